@@ -1,0 +1,295 @@
+"""Focus oracle -- TEST INFRASTRUCTURE, not part of the product.
+
+Python face of the fp64 CPU oracle.  The per-row attention and the group assignment are the C
+functions in ``focus_oracle.c`` (called through ctypes); the remaining pieces are plain numpy.
+Nothing here imports, links or shares code with the CUDA library, and the product never imports
+this module: only the tests, the smoke check and the bench's CPU-baseline leg do.
+
+Passages of the paper each function follows:
+
+* ``assign``            Sec. 2 "Learned grouping" (Eq. 1) + the top-k membership rule of Sec. 2
+                        "Efficiency at inference" and Sec. 3.6.
+* ``attn_rows``         Sec. 2 (exact softmax over attended pairs) + Appendix C, first equation
+                        (the hard Focus mask), with "same group" read as "membership sets intersect".
+* ``dense_brute``       the O(n^2) masked reference the paper verifies against (Appendix C,
+                        "Empirical verification"): explicit n x n boolean matrix, textbook softmax.
+* ``ab_merge``          Appendix C "Disjoint decomposition" and "Merge": sets A (same-group causal)
+                        and B (cross-group local) computed separately and joined through their
+                        logsumexps.  Defined by the paper for single-group assignment only.
+* ``kept_pairs``        size of the attended set of Appendix C's mask (exact integer count).
+* ``tile_reference``    the per-tile mask summaries and the far-tile liveness rule (a far tile can be
+                        dropped when no query of the tile shares a group with any key of the tile);
+                        this is the tile-level consequence of Sec. 2 "different-group distant pairs
+                        are never computed".
+* ``class_sort``        Sec. 2 "Sort tokens by group (stable sort preserves causal order)".
+
+Parity status: every function above is pinned by the CPU tests.  "parity unpinned": the paper's
+perplexity and benchmark numbers (datasets and trained weights are not available).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "focus_oracle.c")
+_LIB = os.path.join(_HERE, "libfocus_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile focus_oracle.c with gcc into libfocus_oracle.so beside it."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c99", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB)
+        c_i64, c_int, c_dbl, vp = ctypes.c_int64, ctypes.c_int, ctypes.c_double, ctypes.c_void_p
+        lib.focus_oracle_threads.restype = c_int
+        lib.focus_oracle_assign.restype = c_int
+        lib.focus_oracle_assign.argtypes = [vp, c_int, c_int, c_i64, c_int, vp, c_int, c_int, vp, vp]
+        lib.focus_oracle_attn_rows.restype = c_int
+        lib.focus_oracle_attn_rows.argtypes = [vp, vp, vp, c_int, c_int, c_i64, c_int, vp, vp, c_i64,
+                                               c_dbl, c_dbl, c_i64, vp, vp, vp, vp, vp, vp]
+        _lib = lib
+    return _lib
+
+
+def threads() -> int:
+    return int(_load().focus_oracle_threads())
+
+
+def _ptr(a):
+    return a.ctypes.data_as(ctypes.c_void_p) if a is not None else None
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """bf16 bit patterns (uint16) -> float64, exactly."""
+    u = bits.astype(np.uint32) << 16
+    return u.view(np.float32).astype(np.float64)
+
+
+def assign(x_bits: np.ndarray, centroids: np.ndarray, topk: int):
+    """x_bits uint16 [H, n, D], centroids float32 [Hkv, K, D] -> (masks uint32 [H, n], margins f64 [H, n])."""
+    x_bits = _c(x_bits, np.uint16)
+    centroids = _c(centroids, np.float32)
+    H, n, D = x_bits.shape
+    Hkv, K, D2 = centroids.shape
+    assert D2 == D
+    masks = np.zeros((H, n), np.uint32)
+    margins = np.zeros((H, n), np.float64)
+    rc = _load().focus_oracle_assign(_ptr(x_bits), H, Hkv, n, D, _ptr(centroids), K, topk,
+                                     _ptr(masks), _ptr(margins))
+    if rc != 0:
+        raise ValueError("focus_oracle_assign: bad arguments")
+    return masks, margins
+
+
+def attn_rows(q_bits, k_bits, v_bits, mq, mk, window, scale=None, softcap=0.0, rows=None):
+    """Attention rows from the definition.
+
+    q_bits uint16 [Hq, n, D]; k_bits, v_bits uint16 [Hkv, n, D]; mq uint32 [Hq, n]; mk uint32 [Hkv, n].
+    rows: int array [R, 2] of (head, token) pairs, or None for every row (head-major order).
+    Returns dict(O f64 [R, D], lse f64 [R], psum f64 [R], kept int64 [R], rows [R, 2]).
+    """
+    q_bits = _c(q_bits, np.uint16); k_bits = _c(k_bits, np.uint16); v_bits = _c(v_bits, np.uint16)
+    mq = _c(mq, np.uint32); mk = _c(mk, np.uint32)
+    Hq, n, D = q_bits.shape
+    Hkv = k_bits.shape[0]
+    assert k_bits.shape == (Hkv, n, D) and v_bits.shape == (Hkv, n, D)
+    assert mq.shape == (Hq, n) and mk.shape == (Hkv, n)
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    if rows is None:
+        hh, ii = np.meshgrid(np.arange(Hq), np.arange(n), indexing="ij")
+        rows = np.stack([hh.ravel(), ii.ravel()], axis=1)
+    rows = np.asarray(rows, dtype=np.int64).reshape(-1, 2)
+    R = rows.shape[0]
+    row_h = _c(rows[:, 0], np.int32); row_i = _c(rows[:, 1], np.int64)
+    O = np.zeros((R, D), np.float64); lse = np.zeros(R, np.float64)
+    psum = np.zeros(R, np.float64); kept = np.zeros(R, np.int64)
+    rc = _load().focus_oracle_attn_rows(_ptr(q_bits), _ptr(k_bits), _ptr(v_bits), Hq, Hkv, n, D,
+                                        _ptr(mq), _ptr(mk), int(window), float(scale), float(softcap),
+                                        R, _ptr(row_h), _ptr(row_i), _ptr(O), _ptr(lse), _ptr(psum),
+                                        _ptr(kept))
+    if rc != 0:
+        raise ValueError("focus_oracle_attn_rows: bad arguments")
+    return dict(O=O, lse=lse, psum=psum, kept=kept, rows=rows)
+
+
+# ----------------------------------------------------------------------------------------------
+# numpy pieces
+# ----------------------------------------------------------------------------------------------
+
+def kept_matrix(mq_h: np.ndarray, mk_h: np.ndarray, window: int) -> np.ndarray:
+    """Explicit n x n boolean mask of Appendix C's first equation for one (q head, kv head) pair."""
+    n = mq_h.shape[0]
+    i = np.arange(n)[:, None]
+    j = np.arange(n)[None, :]
+    share = (mq_h[:, None] & mk_h[None, :]) != 0
+    return (j <= i) & (((i - j) <= window) | share)
+
+
+def dense_brute(q_bits, k_bits, v_bits, mq, mk, window, scale=None, softcap=0.0):
+    """O(n^2) masked reference: explicit mask, -inf elsewhere, full-row textbook softmax, times V.
+
+    Returns (O f64 [Hq, n, D], lse f64 [Hq, n]).  Small n only.
+    """
+    Hq, n, D = q_bits.shape
+    Hkv = k_bits.shape[0]
+    G = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    Q = bf16_bits_to_f64(np.asarray(q_bits)); Kd = bf16_bits_to_f64(np.asarray(k_bits))
+    V = bf16_bits_to_f64(np.asarray(v_bits))
+    O = np.zeros((Hq, n, D)); L = np.zeros((Hq, n))
+    for h in range(Hq):
+        hk = h // G
+        S = scale * (Q[h] @ Kd[hk].T)
+        if softcap > 0:
+            S = softcap * np.tanh(S / softcap)
+        M = kept_matrix(np.asarray(mq)[h], np.asarray(mk)[hk], window)
+        S = np.where(M, S, -np.inf)
+        mx = S.max(axis=1, keepdims=True)
+        E = np.exp(S - mx)
+        Z = E.sum(axis=1, keepdims=True)
+        O[h] = (E / Z) @ V[hk]
+        L[h] = (mx + np.log(Z))[:, 0]
+    return O, L
+
+
+def ab_merge(q_bits, k_bits, v_bits, g, window, scale=None, double_count=False):
+    """Appendix C two-set path for single-group assignment g [n] (one head, MHA).
+
+    Set A = same-group causal pairs, set B = cross-group pairs inside the window; each set gets its
+    own softmax attention and logsumexp, joined by the Appendix C merge formula.  With
+    ``double_count=True`` set B is replaced by *all* local pairs (the overlapping decomposition the
+    paper rejects), which counts same-group local pairs twice.
+    q_bits/k_bits/v_bits uint16 [n, D].  Returns (O [n, D], lse [n]).
+    """
+    n, D = q_bits.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    Q = bf16_bits_to_f64(q_bits); Kd = bf16_bits_to_f64(k_bits); V = bf16_bits_to_f64(v_bits)
+    S = scale * (Q @ Kd.T)
+    i = np.arange(n)[:, None]; j = np.arange(n)[None, :]
+    causal = j <= i
+    same = g[:, None] == g[None, :]
+    local = (i - j) <= window
+    A = causal & same
+    B = causal & local & (np.ones_like(same) if double_count else ~same)
+
+    def part(M):
+        Sm = np.where(M, S, -np.inf)
+        mx = Sm.max(axis=1, keepdims=True)
+        has = np.isfinite(mx)
+        mx0 = np.where(has, mx, 0.0)
+        E = np.where(M, np.exp(Sm - mx0), 0.0)
+        Z = E.sum(axis=1, keepdims=True)
+        o = np.where(has, (E @ V) / np.where(Z > 0, Z, 1.0), 0.0)
+        l = np.where(has[:, 0], mx0[:, 0] + np.log(np.where(Z[:, 0] > 0, Z[:, 0], 1.0)), -np.inf)
+        return o, l
+
+    oA, lA = part(A)
+    oB, lB = part(B)
+    mx = np.maximum(lA, lB)
+    eA = np.exp(lA - mx); eB = np.exp(lB - mx)
+    O = (eA[:, None] * oA + eB[:, None] * oB) / (eA + eB)[:, None]
+    return O, mx + np.log(eA + eB)
+
+
+def kept_pairs(mq: np.ndarray, mk: np.ndarray, window: int) -> np.ndarray:
+    """Exact number of attended pairs per query head (int64 [Hq]).
+
+    Row i keeps its min(i, w) + 1 local keys plus every key j < i - w whose membership mask meets
+    the row's; the second term is read from a running count of far keys per distinct key mask.
+    """
+    mq = np.asarray(mq, np.uint32); mk = np.asarray(mk, np.uint32)
+    Hq, n = mq.shape
+    Hkv = mk.shape[0]
+    G = Hq // Hkv
+    out = np.zeros(Hq, np.int64)
+    idx = np.arange(n, dtype=np.int64)
+    far_len = np.maximum(idx - window, 0)            # number of keys j with i - j > w
+    local = np.minimum(idx, window) + 1
+    for h in range(Hq):
+        hk = h // G
+        total = int(local.sum())
+        kvals = np.unique(mk[hk])
+        for qv in np.unique(mq[h]):
+            sharing = kvals[(kvals & qv) != 0]
+            if sharing.size == 0:
+                continue
+            is_share = np.isin(mk[hk], sharing)
+            cum = np.concatenate([[0], np.cumsum(is_share, dtype=np.int64)])   # cum[m] = # sharing keys j < m
+            rows = mq[h] == qv
+            total += int(cum[far_len[rows]].sum())
+        out[h] = total
+    return out
+
+
+def tile_reference(mq: np.ndarray, mk: np.ndarray, window: int, BM: int, BN: int):
+    """Tile summaries and far-tile liveness, straight from their definitions.
+
+    Query tile a covers rows [a*BM, min(n, (a+1)*BM)), key tile b covers keys [b*BN, min(n, (b+1)*BN)).
+    Returns dict with
+      orq, andq  uint32 [Hq, nqt]   OR / AND of the member masks of each query tile
+      ork, andk  uint32 [Hkv, nkt]
+      far        bool [nqt, nkt]    every pair of the tile pair has i - j > w (so it is causal too)
+      live       bool [Hq, nqt, nkt] far and (orq & ork != 0)
+      full       bool [Hq, nqt, nkt] far and (andq & andk != 0): every pair shares a group
+    """
+    mq = np.asarray(mq, np.uint32); mk = np.asarray(mk, np.uint32)
+    Hq, n = mq.shape
+    Hkv = mk.shape[0]
+    G = Hq // Hkv
+    nqt = (n + BM - 1) // BM
+    nkt = (n + BN - 1) // BN
+
+    def summarise(m, T, nt):
+        o = np.zeros((m.shape[0], nt), np.uint32); a = np.zeros((m.shape[0], nt), np.uint32)
+        for t in range(nt):
+            seg = m[:, t * T:min(n, (t + 1) * T)]
+            o[:, t] = np.bitwise_or.reduce(seg, axis=1)
+            a[:, t] = np.bitwise_and.reduce(seg, axis=1)
+        return o, a
+
+    orq, andq = summarise(mq, BM, nqt)
+    ork, andk = summarise(mk, BN, nkt)
+    qmin = np.arange(nqt) * BM
+    kmax = np.minimum(n, (np.arange(nkt) + 1) * BN) - 1
+    far = (qmin[:, None] - kmax[None, :]) > window
+    live = np.zeros((Hq, nqt, nkt), bool); full = np.zeros((Hq, nqt, nkt), bool)
+    for h in range(Hq):
+        hk = h // G
+        live[h] = far & ((orq[h][:, None] & ork[hk][None, :]) != 0)
+        full[h] = far & ((andq[h][:, None] & andk[hk][None, :]) != 0)
+    return dict(orq=orq, andq=andq, ork=ork, andk=andk, far=far, live=live, full=full)
+
+
+def class_sort(m_h: np.ndarray):
+    """Stable sort of one head's tokens by membership-mask value.
+
+    Returns (perm int64 [n], classes uint32 [C], counts int64 [C]): perm lists original positions,
+    class by class (classes ascending by mask value), positions ascending inside a class.
+    """
+    m_h = np.asarray(m_h, np.uint32)
+    perm = np.argsort(m_h, kind="stable").astype(np.int64)
+    classes, counts = np.unique(m_h, return_counts=True)
+    return perm, classes.astype(np.uint32), counts.astype(np.int64)

@@ -1,0 +1,362 @@
+"""Pins for the CPU oracle: each test ties an oracle function to something other than itself --
+an explicit dense-mask brute force, a library routine (torch SDPA / cosine_similarity / topk),
+a closed form, a value printed in the paper, or a case worked by hand."""
+import math
+import os
+from math import comb
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import focus_oracle as fo
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bits(x):
+    """float array -> bf16 bit patterns (RNE) via torch."""
+    t = torch.as_tensor(np.asarray(x, dtype=np.float32)).to(torch.bfloat16)
+    return t.view(torch.int16).numpy().view(np.uint16)
+
+
+def rand_bits(rng, shape):
+    return bits(rng.standard_normal(shape))
+
+
+def rand_masks(rng, H, n, K, t):
+    """uniform random t-subsets of K groups as bit masks"""
+    out = np.zeros((H, n), np.uint32)
+    for h in range(H):
+        for i in range(n):
+            out[h, i] = sum(1 << int(g) for g in rng.choice(K, size=t, replace=False))
+    return out
+
+
+def sdpa_causal(qb, kb, vb, scale):
+    """library reference: torch scaled_dot_product_attention, causal, fp64, GQA by repeating KV heads"""
+    Q = torch.from_numpy(fo.bf16_bits_to_f64(qb)); K = torch.from_numpy(fo.bf16_bits_to_f64(kb))
+    V = torch.from_numpy(fo.bf16_bits_to_f64(vb))
+    G = Q.shape[0] // K.shape[0]
+    K = K.repeat_interleave(G, dim=0); V = V.repeat_interleave(G, dim=0)
+    return torch.nn.functional.scaled_dot_product_attention(Q, K, V, is_causal=True, scale=scale).numpy()
+
+
+# ------------------------------------------------------------------------------------------------
+# attention rows
+# ------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n", [1, 2, 3, 17, 64, 129, 257])
+@pytest.mark.parametrize("Hq,Hkv,D", [(2, 2, 8), (4, 2, 16), (6, 2, 64)])
+def test_rows_vs_dense_bruteforce(n, Hq, Hkv, D):
+    """explicit n x n mask + textbook softmax (numpy) == row-by-row C oracle"""
+    rng = np.random.default_rng(n * 131 + Hq * 7 + D)
+    K = int(rng.choice([2, 4, 8])); t = int(rng.integers(1, K + 1)); w = int(rng.integers(0, n + 2))
+    softcap = float(rng.choice([0.0, 3.0]))
+    q = rand_bits(rng, (Hq, n, D)); k = rand_bits(rng, (Hkv, n, D)); v = rand_bits(rng, (Hkv, n, D))
+    mq = rand_masks(rng, Hq, n, K, t); mk = rand_masks(rng, Hkv, n, K, t)
+    r = fo.attn_rows(q, k, v, mq, mk, w, softcap=softcap)
+    O, L = fo.dense_brute(q, k, v, mq, mk, w, softcap=softcap)
+    np.testing.assert_allclose(r["O"].reshape(Hq, n, D), O, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(r["lse"].reshape(Hq, n), L, rtol=0, atol=1e-12)
+    # kept counter against the explicit matrix
+    G = Hq // Hkv
+    cnt = np.stack([fo.kept_matrix(mq[h], mk[h // G], w).sum(axis=1) for h in range(Hq)])
+    assert np.array_equal(r["kept"].reshape(Hq, n), cnt)
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(3, 3), (8, 2)])
+def test_window_covers_sequence_is_plain_causal(Hq, Hkv):
+    """w >= n: every causal pair is local, so the result is textbook causal attention (torch SDPA),
+    whatever the masks say.  With GQA this also pins 'consecutive query heads share a KV head'."""
+    rng = np.random.default_rng(5)
+    n, D = 96, 32
+    q = rand_bits(rng, (Hq, n, D)); k = rand_bits(rng, (Hkv, n, D)); v = rand_bits(rng, (Hkv, n, D))
+    mq = rand_masks(rng, Hq, n, 4, 1); mk = rand_masks(rng, Hkv, n, 4, 1)
+    ref = sdpa_causal(q, k, v, 1.0 / math.sqrt(D))
+    for w in (n, n + 7, 10 * n):
+        r = fo.attn_rows(q, k, v, mq, mk, w)
+        np.testing.assert_allclose(r["O"].reshape(Hq, n, D), ref, rtol=0, atol=1e-12)
+
+
+def test_single_group_is_plain_causal():
+    """K = 1: assignment puts every token in group 0, every pair shares it -> full causal attention"""
+    rng = np.random.default_rng(6)
+    Hq, Hkv, n, D = 4, 2, 80, 16
+    q = rand_bits(rng, (Hq, n, D)); k = rand_bits(rng, (Hkv, n, D)); v = rand_bits(rng, (Hkv, n, D))
+    C = rng.standard_normal((Hkv, 1, D)).astype(np.float32)
+    mq, _ = fo.assign(q, C, 1); mk, _ = fo.assign(k, C, 1)
+    assert (mq == 1).all() and (mk == 1).all()
+    r = fo.attn_rows(q, k, v, mq, mk, 0)
+    np.testing.assert_allclose(r["O"].reshape(Hq, n, D), sdpa_causal(q, k, v, 1.0 / math.sqrt(D)), atol=1e-12)
+
+
+@pytest.mark.parametrize("K,t", [(4, 3), (4, 4), (8, 5), (2, 2)])
+def test_pigeonhole_topk_is_plain_causal(K, t):
+    """2t > K: any two t-subsets intersect, so nothing is pruned.  The paper's top-k table prints 100 %
+    pairs retained for k = 3 and k = 4 of K = 4."""
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "paper_topk_table.txt")) if not l.startswith("#")]
+    for model, k, _, pct in rows:
+        if int(k) >= 3:
+            assert int(pct) == 100
+    rng = np.random.default_rng(K * 10 + t)
+    Hq = Hkv = 2; n = 70; D = 8
+    q = rand_bits(rng, (Hq, n, D)); k = rand_bits(rng, (Hkv, n, D)); v = rand_bits(rng, (Hkv, n, D))
+    mq = rand_masks(rng, Hq, n, K, t); mk = rand_masks(rng, Hkv, n, K, t)
+    r = fo.attn_rows(q, k, v, mq, mk, 0)
+    np.testing.assert_allclose(r["O"].reshape(Hq, n, D), sdpa_causal(q, k, v, 1.0 / math.sqrt(D)), atol=1e-12)
+    assert np.array_equal(fo.kept_pairs(mq, mk, 0), np.full(Hq, n * (n + 1) // 2))
+
+
+def test_rows_are_stochastic_and_lse_is_log_partition():
+    rng = np.random.default_rng(8)
+    Hq, Hkv, n, D = 4, 2, 150, 16
+    q = rand_bits(rng, (Hq, n, D)); k = rand_bits(rng, (Hkv, n, D)); v = rand_bits(rng, (Hkv, n, D))
+    mq = rand_masks(rng, Hq, n, 4, 2); mk = rand_masks(rng, Hkv, n, 4, 2)
+    r = fo.attn_rows(q, k, v, mq, mk, 9)
+    np.testing.assert_allclose(r["psum"], 1.0, atol=1e-12)
+    # V = all-ones -> every output coordinate equals the total weight 1
+    ones = bits(np.ones((Hkv, n, D)))
+    r1 = fo.attn_rows(q, k, ones, mq, mk, 9)
+    np.testing.assert_allclose(r1["O"], 1.0, atol=1e-12)
+    # exp(lse) is the unnormalised partition sum: check through torch.logsumexp on the kept logits
+    Q = fo.bf16_bits_to_f64(q); Kd = fo.bf16_bits_to_f64(k)
+    for (h, i) in [(0, 0), (1, 37), (3, 149)]:
+        keep = fo.kept_matrix(mq[h], mk[h // 2], 9)[i]
+        s = (Q[h, i] @ Kd[h // 2].T) / math.sqrt(D)
+        ref = torch.logsumexp(torch.from_numpy(s[keep]), 0).item()
+        assert abs(r["lse"][h * n + i] - ref) < 1e-12
+
+
+def test_hand_worked_case():
+    """n=4, D=2, K=2 groups, top-1, w=1, scale=1; everything below is worked by hand.
+
+    centroids c0=(1,0), c1=(0,1).  x0=(1,0)->g0, x1=(0,1)->g1, x2=(0,2)->g1, x3=(2,0)->g0 (Q = K = x).
+    kept sets: row0 {0}; row1 {0 (local), 1}; row2 {1 (local), 2}  (0 is 2 away and in another group);
+    row3 {0 (far, same group), 2 (local, other group), 3}  (1 is 2 away and in another group).
+    """
+    x = np.array([[1, 0], [0, 1], [0, 2], [2, 0]], np.float32)[None]
+    V = np.array([[1, 0], [0, 1], [1, 1], [-1, 2]], np.float32)[None]
+    C = np.array([[[1, 0], [0, 1]]], np.float32)
+    m, margins = fo.assign(bits(x), C, 1)
+    assert m.tolist() == [[1, 2, 2, 1]]
+    np.testing.assert_allclose(margins, 1.0, atol=1e-15)        # cosines are exactly 1 and 0
+    r = fo.attn_rows(bits(x), bits(x), bits(V), m, m, 1, scale=1.0)
+    e = math.exp
+    O = r["O"]; L = r["lse"]
+    assert r["kept"].tolist() == [1, 2, 2, 3]
+    np.testing.assert_allclose(O[0], [1, 0], atol=1e-15); assert abs(L[0] - 1.0) < 1e-15
+    # row1: s10 = 0, s11 = 1
+    np.testing.assert_allclose(O[1], [1 / (1 + e(1)), e(1) / (1 + e(1))], atol=1e-15)
+    assert abs(L[1] - math.log(1 + e(1))) < 1e-15
+    # row2: s21 = 2, s22 = 4
+    z = e(2) + e(4)
+    np.testing.assert_allclose(O[2], [e(4) / z, (e(2) + e(4)) / z], atol=1e-15)
+    assert abs(L[2] - math.log(z)) < 1e-14
+    # row3: s30 = 2, s32 = 0, s33 = 4
+    z = e(2) + 1 + e(4)
+    np.testing.assert_allclose(O[3], [(e(2) + 1 - e(4)) / z, (1 + 2 * e(4)) / z], atol=1e-15)
+    assert abs(L[3] - math.log(z)) < 1e-14
+    # w = 0 drops the distance-1 neighbours of other groups; w = 2 brings back (2,0) and (3,1)
+    assert fo.attn_rows(bits(x), bits(x), bits(V), m, m, 0, scale=1.0)["kept"].tolist() == [1, 1, 2, 2]
+    assert fo.attn_rows(bits(x), bits(x), bits(V), m, m, 2, scale=1.0)["kept"].tolist() == [1, 2, 3, 4]
+
+
+def test_softcap_closed_form_and_limit():
+    """two keys: weight ratio is exp(c*tanh(s1/c) - c*tanh(s0/c)); a huge cap changes nothing"""
+    q = np.array([[[0, 0], [3, 1]]], np.float32); k = np.array([[[2, 0], [1, 3]]], np.float32)
+    v = np.array([[[1, 0], [0, 1]]], np.float32)
+    m = np.ones((1, 2), np.uint32)
+    c = 2.0
+    r = fo.attn_rows(bits(q), bits(k), bits(v), m, m, 5, scale=0.5, softcap=c)
+    s0 = c * math.tanh(0.5 * 6 / c); s1 = c * math.tanh(0.5 * 6 / c)
+    assert s0 == s1
+    np.testing.assert_allclose(r["O"][1], [0.5, 0.5], atol=1e-15)
+    k2 = np.array([[[2, 0], [1, 1]]], np.float32)                 # s0 = 3, s1 = 2 before capping
+    r = fo.attn_rows(bits(q), bits(k2), bits(v), m, m, 5, scale=0.5, softcap=c)
+    a, b = c * math.tanh(3 / c), c * math.tanh(2 / c)
+    np.testing.assert_allclose(r["O"][1], [math.exp(a) / (math.exp(a) + math.exp(b)),
+                                           math.exp(b) / (math.exp(a) + math.exp(b))], atol=1e-15)
+    assert abs(r["lse"][1] - math.log(math.exp(a) + math.exp(b))) < 1e-15
+    rng = np.random.default_rng(3)
+    qq = rand_bits(rng, (2, 40, 8)); kk = rand_bits(rng, (2, 40, 8)); vv = rand_bits(rng, (2, 40, 8))
+    mm = rand_masks(rng, 2, 40, 4, 2)
+    big = fo.attn_rows(qq, kk, vv, mm, mm, 4, softcap=1e9)["O"]
+    off = fo.attn_rows(qq, kk, vv, mm, mm, 4, softcap=0.0)["O"]
+    np.testing.assert_allclose(big, off, atol=1e-9)
+
+
+def test_two_set_merge_matches_and_double_count_fails():
+    """Appendix C: sets A (same-group causal) and B (cross-group local) merged through their
+    logsumexps equal the masked definition (the paper reports cosine similarity 1.0000); the
+    overlapping same-group + all-local split double counts and must NOT match."""
+    rng = np.random.default_rng(11)
+    n, D, K, w = 200, 16, 4, 12
+    q = rand_bits(rng, (n, D)); k = rand_bits(rng, (n, D)); v = rand_bits(rng, (n, D))
+    g = rng.integers(0, K, n)
+    m = (1 << g).astype(np.uint32)[None]
+    ref = fo.attn_rows(q[None], k[None], v[None], m, m, w)
+    O, L = fo.ab_merge(q, k, v, g, w)
+    np.testing.assert_allclose(O, ref["O"], atol=1e-12)
+    np.testing.assert_allclose(L, ref["lse"], atol=1e-12)
+
+    def cos(a, b):
+        return float((a * b).sum() / np.sqrt((a * a).sum() * (b * b).sum()))
+
+    assert round(cos(O, ref["O"]), 4) == 1.0
+    Obad, _ = fo.ab_merge(q, k, v, g, w, double_count=True)
+    assert np.abs(Obad - ref["O"]).max() > 1e-2
+    assert cos(Obad, ref["O"]) < 0.9999
+
+
+# ------------------------------------------------------------------------------------------------
+# kept-pair counts
+# ------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n,w", [(1, 0), (33, 0), (130, 7), (257, 300)])
+def test_kept_pairs_vs_explicit_matrix(n, w):
+    rng = np.random.default_rng(n + w)
+    Hq, Hkv = 4, 2
+    mq = rand_masks(rng, Hq, n, 8, 2); mk = rand_masks(rng, Hkv, n, 8, 2)
+    want = [int(fo.kept_matrix(mq[h], mk[h // 2], w).sum()) for h in range(Hq)]
+    assert fo.kept_pairs(mq, mk, w).tolist() == want
+
+
+@pytest.mark.parametrize("K,t", [(4, 1), (4, 2), (8, 2), (8, 1)])
+def test_far_kept_fraction_closed_form(K, t):
+    """independent uniform t-subsets share a group with probability 1 - C(K-t,t)/C(K,t); for t = 1
+    this is the paper's 1/K (n^2/K cost; 25-26 % of pairs retained at K=4, k=1 in its top-k table)."""
+    if t == 1:
+        model = {int(l.split()[0]): float(l.split()[1])
+                 for l in open(os.path.join(GOLDEN, "paper_speedup_model.txt")) if not l.startswith("#")}
+        assert abs(model[K] - (1 - comb(K - t, t) / comb(K, t))) < 1e-15
+    if (K, t) == (4, 1):
+        tab = [l.split() for l in open(os.path.join(GOLDEN, "paper_topk_table.txt")) if not l.startswith("#")]
+        assert all(abs(int(p) - 25) <= 1 for _, k, _, p in tab if int(k) == 1)
+    rng = np.random.default_rng(K * 100 + t)
+    n = 3000
+    mq = rand_masks(rng, 1, n, K, t); mk = rand_masks(rng, 1, n, K, t)
+    far_total = n * (n + 1) // 2 - n                          # w = 0: only the diagonal is local
+    frac = (int(fo.kept_pairs(mq, mk, 0)[0]) - n) / far_total
+    want = 1 - comb(K - t, t) / comb(K, t)
+    assert abs(frac - want) < 4 * math.sqrt(want * (1 - want) / n)   # rows are the independent units
+
+
+# ------------------------------------------------------------------------------------------------
+# assignment
+# ------------------------------------------------------------------------------------------------
+
+def test_assign_matches_library_cosine_topk():
+    """torch cosine_similarity + topk in fp64 as the library reference (no exact ties in random data)"""
+    rng = np.random.default_rng(21)
+    H, Hkv, n, D, K, t = 6, 3, 300, 32, 8, 3
+    x = rand_bits(rng, (H, n, D))
+    C = rng.standard_normal((Hkv, K, D)).astype(np.float32) * rng.uniform(0.5, 3, (Hkv, K, 1)).astype(np.float32)
+    masks, margins = fo.assign(x, C, t)
+    X = torch.from_numpy(fo.bf16_bits_to_f64(x))
+    Ct = torch.from_numpy(C.astype(np.float64)).repeat_interleave(H // Hkv, dim=0)      # [H, K, D]
+    cs = torch.nn.functional.cosine_similarity(X[:, :, None, :], Ct[:, None, :, :], dim=-1, eps=0)
+    top = torch.topk(cs, t + 1, dim=-1)
+    want = (1 << top.indices[..., :t]).sum(-1).numpy().astype(np.uint32)
+    assert np.array_equal(masks, want)
+    np.testing.assert_allclose(margins, (top.values[..., t - 1] - top.values[..., t]).numpy(), atol=1e-14)
+
+
+def test_assign_geometry_ties_scaling():
+    # D = 2, centroids at 0, 90, 180 degrees (non-unit lengths: cosine ignores them)
+    C = np.array([[[3, 0], [0, 0.5], [-2, 0]]], np.float32)
+    ang = np.deg2rad([10, 80, 100, 170, 44, 46])
+    x = np.stack([np.cos(ang), np.sin(ang)], 1).astype(np.float32)[None] * 4
+    m, mg = fo.assign(bits(x), C, 1)
+    assert m.tolist() == [[1, 2, 2, 4, 1, 2]]
+    m2, _ = fo.assign(bits(x), C, 2)
+    assert m2.tolist() == [[3, 3, 6, 6, 3, 3]]
+    # margin for the 10-degree vector at t=1: cos(10deg) - cos(80deg), up to bf16 rounding of x
+    xb = fo.bf16_bits_to_f64(bits(x))[0, 0]
+    a = math.atan2(xb[1], xb[0])
+    assert abs(mg[0, 0] - (math.cos(a) - math.cos(math.pi / 2 - a))) < 1e-12
+    # exact ties: duplicate centroids -> lower index wins; zero vector -> groups 0..t-1
+    Cd = np.array([[[1, 1], [1, 1], [1, 1], [-1, 0]]], np.float32)
+    z = np.array([[[2, 2], [0, 0], [-1, 0]]], np.float32)
+    m, mg = fo.assign(bits(z), Cd, 2)
+    assert m.tolist() == [[0b0011, 0b0011, 0b1001]]
+    assert mg[0, 0] == 0.0 and mg[0, 1] == 0.0
+    # positive rescaling of tokens (exact in bf16) and of centroids changes nothing; t = K margin is inf
+    rng = np.random.default_rng(2)
+    xr = rng.standard_normal((2, 50, 16)).astype(np.float32)
+    Cr = rng.standard_normal((2, 4, 16)).astype(np.float32)
+    a, _ = fo.assign(bits(xr), Cr, 2)
+    b, _ = fo.assign(bits(bits_scale(xr, 4.0)), Cr * np.float32(0.125), 2)
+    assert np.array_equal(a, b)
+    full, mg = fo.assign(bits(xr), Cr, 4)
+    assert (full == 15).all() and np.isinf(mg).all()
+
+
+def bits_scale(x, s):
+    return fo.bf16_bits_to_f64(bits(x)).astype(np.float32) * np.float32(s)
+
+
+def test_assign_dominant_centroid():
+    """x = 5*c_g + small noise must land in group g first"""
+    rng = np.random.default_rng(4)
+    Hkv, K, D = 2, 8, 64
+    C = rng.standard_normal((Hkv, K, D)).astype(np.float32)
+    C /= np.linalg.norm(C, axis=-1, keepdims=True)
+    g = rng.integers(0, K, (4, 100))
+    x = 5 * C[np.arange(4)[:, None] // 2, g] + 0.1 * rng.standard_normal((4, 100, D)).astype(np.float32)
+    m, _ = fo.assign(bits(x), C, 1)
+    assert np.array_equal(m, (1 << g).astype(np.uint32))
+
+
+# ------------------------------------------------------------------------------------------------
+# tile summaries and class sort
+# ------------------------------------------------------------------------------------------------
+
+def test_tile_reference_is_sound_and_tight():
+    """a far tile pair is dead exactly when the explicit mask has no kept pair in it (given w), and
+    'full' tiles are entirely kept"""
+    rng = np.random.default_rng(31)
+    Hq, Hkv, n, BM, BN, w = 2, 1, 200, 16, 8, 10
+    # few groups per tile so that some tiles really die: group depends on position block
+    blk = (np.arange(n) // 24) % 4
+    mk = (1 << blk).astype(np.uint32)[None]
+    mq = np.stack([(1 << blk), (1 << ((blk + (np.arange(n) % 7 == 0)) % 4))]).astype(np.uint32)
+    ref = fo.tile_reference(mq, mk, w, BM, BN)
+    nqt, nkt = ref["far"].shape
+    dead_seen = live_seen = full_seen = 0
+    for h in range(Hq):
+        M = fo.kept_matrix(mq[h], mk[0], w)
+        for a in range(nqt):
+            for b in range(nkt):
+                rows = slice(a * BM, min(n, (a + 1) * BM)); cols = slice(b * BN, min(n, (b + 1) * BN))
+                sub = M[rows, cols]
+                i = np.arange(n)[rows][:, None]; j = np.arange(n)[cols][None, :]
+                is_far = bool(((i - j) > w).all())
+                assert ref["far"][a, b] == is_far
+                if is_far and not ref["live"][h, a, b]:
+                    assert not sub.any(); dead_seen += 1
+                if ref["live"][h, a, b]:
+                    live_seen += 1
+                if ref["full"][h, a, b]:
+                    assert sub.all() and ref["live"][h, a, b]; full_seen += 1
+    assert dead_seen > 0 and live_seen > 0 and full_seen > 0
+
+
+def test_class_sort_is_stable_and_preserves_kept_sets():
+    """sorting tokens by mask value with a stable sort keeps positions ascending inside a class, and
+    the kept rule evaluated on (sorted index -> original position) is the same set of pairs"""
+    rng = np.random.default_rng(41)
+    n, w = 300, 9
+    mq = rand_masks(rng, 1, n, 4, 2)[0]; mk = rand_masks(rng, 1, n, 4, 2)[0]
+    pq, cq, nq = fo.class_sort(mq); pk, ck, nk = fo.class_sort(mk)
+    assert sorted(pq.tolist()) == list(range(n)) and nq.sum() == n
+    off = 0
+    for c, cnt in zip(cq, nq):
+        seg = pq[off:off + cnt]
+        assert (mq[seg] == c).all() and (np.diff(seg) > 0).all()
+        off += cnt
+    M = fo.kept_matrix(mq, mk, w)
+    posq = pq[:, None]; posk = pk[None, :]
+    share = (mq[pq][:, None] & mk[pk][None, :]) != 0
+    Ms = (posk <= posq) & (((posq - posk) <= w) | share)
+    assert np.array_equal(Ms, M[np.ix_(pq, pk)])
