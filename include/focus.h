@@ -1,0 +1,196 @@
+/*
+ * focus.h -- C ABI of the Focus inference hot path for NVIDIA B200 (sm_100a).
+ *
+ * Focus (arXiv 2604.03260, "Composing Sparse Attention via Learned Grouping") restricts causal
+ * attention to pairs that are close (inside a local window) or that share a learned group, and
+ * keeps exact softmax over the surviving pairs.  This library is the inference path of one
+ * attention layer: group assignment -> tile summaries -> attention forward.
+ *
+ * General rules for every entry point
+ *   - Pointers named "device" must be device memory of the current CUDA device; the caller owns
+ *     every buffer.  The library allocates no device memory.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the legacy default
+ *     stream).  No entry point synchronises the device.
+ *   - Return value: FOCUS_OK (0) or a negative focus_status.  Nothing throws, aborts or traps.
+ *     focus_last_error() gives a thread-local message for the last failure.
+ *   - Tensors are bf16 with the head dimension D contiguous; the other strides are in elements.
+ *     For the attention kernel the base pointer must be 16-byte aligned and every stride a
+ *     multiple of 8 elements (TMA requirements).
+ *   - Query head h uses KV head h / (Hq / Hkv): consecutive query heads share a KV head.
+ *   - Group membership of a token is a uint32 bit mask (bit g = member of group g), K <= 32.
+ */
+#ifndef FOCUS_H_
+#define FOCUS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define FOCUS_API __attribute__((visibility("default")))
+#else
+#define FOCUS_API
+#endif
+
+typedef enum {
+    FOCUS_OK = 0,
+    FOCUS_ERR_INVALID_ARG = -1, /* null pointer, bad size, Hq % Hkv != 0, topk outside [1,K], misaligned tensor */
+    FOCUS_ERR_UNSUPPORTED = -2, /* D not in {64,128,256}, too many mask classes for the sorted layout */
+    FOCUS_ERR_CAPACITY = -3,    /* workspace smaller than focus_tiles_workspace_bytes() */
+    FOCUS_ERR_ARCH = -4,        /* current device is not compute capability 10.x */
+    FOCUS_ERR_CUDA = -5         /* a CUDA call failed; focus_last_error() has its message */
+} focus_status;
+
+/* Problem shape.  batch*Hq query heads and batch*Hkv KV heads of n tokens each. */
+typedef struct {
+    int32_t batch;   /* >= 1 */
+    int32_t Hq;      /* query heads, multiple of Hkv */
+    int32_t Hkv;     /* key/value heads */
+    int32_t n;       /* tokens per sequence, >= 1 */
+    int32_t D;       /* head dimension: 64, 128 or 256 */
+    int32_t K;       /* number of groups, 1..32 */
+    int32_t topk;    /* groups each token joins, 1..K */
+    int32_t window;  /* w >= 0: pairs with i - j <= w are always attended (w+1 keys incl. self) */
+    float scale;     /* logit scale; 0 selects 1/sqrt(D) */
+    float softcap;   /* c > 0: logits become c*tanh(scale*q.k/c) before the softmax; 0 = off */
+} focus_shape;
+
+/* A bf16 tensor [batch, H, n, D] in device memory, D contiguous, strides in elements. */
+typedef struct {
+    void* ptr;
+    int64_t stride_b;
+    int64_t stride_h;
+    int64_t stride_n;
+} focus_tensor;
+
+/* Tile sizes of the summaries written by focus_build_tiles (fixed by the ABI). */
+#define FOCUS_TILE_M 128
+#define FOCUS_TILE_N 128
+/* Largest number of distinct mask values per head the class-sorted layout accepts. */
+#define FOCUS_MAX_CLASSES 64
+
+#define FOCUS_LAYOUT_ORIGINAL 0
+#define FOCUS_LAYOUT_CLASS_SORTED 1
+
+/*
+ * Byte offsets of the arrays inside a tiles workspace (a pure function of shape and layout;
+ * computed on the host, no device access).  nqt = ceil(n/128) query tiles, nkt = ceil(n/128) key
+ * tiles, nkw = ceil(nkt/32).  Heads are indexed batch-major (b*H + h).
+ */
+typedef struct {
+    int32_t layout, nqt, nkt, nkw;
+    size_t total_bytes;
+    size_t counters;   /* uint64[8]: [0] far tile pairs, [1] live far tile pairs, [2] full far tile pairs,
+                                     [3] sorted layout: tile pairs listed in the ranges */
+    size_t orq, andq;  /* uint32 [B*Hq][nqt]: OR / AND of the member masks of each query tile */
+    size_t ork, andk;  /* uint32 [B*Hkv][nkt] */
+    size_t gbits;      /* uint32 [B*Hkv][nkt][K][4]: bit j of word j/32 set when key 128*b + j is in group g */
+    size_t live;       /* uint32 [B*Hq][nqt][nkw]: bit b set when (a, b) is a far tile pair that may hold a kept pair */
+    size_t live_cnt;   /* int32  [B*Hq][nqt]: popcount of the row of `live` */
+    /* class-sorted layout only (0 otherwise) */
+    int32_t nqp, nkp;  /* padded sorted lengths (multiples of 256) */
+    size_t ncls_q, ncls_k;   /* int32 [B*Hq], [B*Hkv]: distinct mask values of the head */
+    size_t cls_q, cls_k;     /* uint32 [heads][FOCUS_MAX_CLASSES]: the mask values, ascending */
+    size_t seg_q, seg_k;     /* int32 [heads][FOCUS_MAX_CLASSES+1]: padded start of each class segment */
+    size_t perm_q, perm_k;   /* int32 [heads][nqp|nkp]: original position of each sorted slot; padding is
+                                -1 on the query side and INT32_MAX on the key side */
+    size_t qrange;           /* int32 [B*Hq][nqp/256][FOCUS_MAX_CLASSES][2]: first and one-past-last sorted
+                                key tile (128 keys) of each key class a 256-row query block must visit */
+    size_t qs, ks, vs;       /* bf16 sorted copies [B*Hq][nqp][D], [B*Hkv][nkp][D] x2 */
+} focus_tiles_layout;
+
+/* Library version (major*10000 + minor*100 + patch). */
+FOCUS_API int focus_version(void);
+FOCUS_API const char* focus_status_string(int status);
+FOCUS_API const char* focus_last_error(void);
+
+/*
+ * focus_assign -- group assignment (paper Sec. 2 "Learned grouping", Eq. 1, with the top-k
+ * membership rule of Sec. 2 "Efficiency at inference" / Sec. 3.6).
+ * For each head vector x (a query head vector or a key head vector) the score against group g
+ * is the cosine between x and centroid g of the vector's KV head; the token joins its `topk` best
+ * groups (ties go to the lower group index; a zero vector scores 0 everywhere).
+ *   x           device, bf16 [batch, H, n, D]
+ *   H           number of heads of x: shape->Hq or shape->Hkv (head h reads centroid set h / (H/Hkv))
+ *   centroids   device, fp32 [Hkv, K, D] contiguous; need not be unit length
+ *   masks_out   device, uint32 [batch*H, n]
+ *   near_ties   device, nullable: *near_ties is incremented (not reset) by the number of vectors whose
+ *               margin cos(topk-th) - cos((topk+1)-th), computed in fp32, is below near_tie_eps
+ * Arithmetic is fp32 on the exact bf16 values.
+ */
+FOCUS_API int focus_assign(const focus_shape* shape, focus_tensor x, int32_t H, const float* centroids,
+                 uint32_t* masks_out, unsigned long long* near_ties, float near_tie_eps, void* stream);
+
+/*
+ * focus_tiles_layout_of -- host-only: sizes and offsets of the tiles workspace.
+ * focus_tiles_workspace_bytes -- its total_bytes (0 on bad arguments).
+ */
+FOCUS_API int focus_tiles_layout_of(const focus_shape* shape, int32_t layout, focus_tiles_layout* out);
+FOCUS_API size_t focus_tiles_workspace_bytes(const focus_shape* shape, int32_t layout);
+
+/*
+ * focus_build_tiles -- per-tile summaries of the membership masks and the live far-tile set
+ * (paper Sec. 2 "Efficiency at inference": different-group distant pairs are never computed;
+ * Sec. 2 item "Group": stable sort of tokens by group for the class-sorted layout).
+ * A tile pair (a, b) is "far" when every pair in it has i - j > w.  A far pair is live iff
+ * OR(query tile masks) & OR(key tile masks) != 0; dead far pairs hold no attended pair.
+ *   mq   device, uint32 [batch*Hq, n]    mk   device, uint32 [batch*Hkv, n]
+ *   layout  FOCUS_LAYOUT_ORIGINAL, or FOCUS_LAYOUT_CLASS_SORTED (tokens stably sorted by mask value
+ *           per head, so that a tile holds one mask class and tile pairs are all-share or none-share)
+ *   ws   device workspace of ws_bytes >= focus_tiles_workspace_bytes(shape, layout), 256-byte aligned.
+ *        Contents are described by focus_tiles_layout.  The workspace is tied to (shape, mq, mk).
+ */
+FOCUS_API int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, const uint32_t* mk, int32_t layout,
+                      void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * focus_attn_fwd -- causal attention forward over the attended pairs (paper Sec. 2 and
+ * Appendix C, first equation): pair (i, j) is attended iff
+ *        j <= i  and  ( i - j <= window  or  mq[h,i] & mk[kv(h),j] != 0 ).
+ * s_ij = scale*q_i.k_j (then softcap*tanh(s_ij/softcap) if softcap > 0);
+ * lse_i = log sum_j exp(s_ij); o_i = sum_j exp(s_ij - lse_i) v_j over attended j: exact softmax,
+ * no renormalisation.  bf16 operands, fp32 accumulation, probabilities rounded to bf16 before PV.
+ *   q, o        device bf16 [batch, Hq, n, D]      k, v   device bf16 [batch, Hkv, n, D]
+ *   mq, mk      device masks; may be NULL when tiles_ws is NULL
+ *   tiles_ws    workspace written by focus_build_tiles for the same shape and masks.  NULL = dense
+ *               causal mode (every causal pair attended; masks and layout ignored).
+ *   layout      the layout the workspace was built with: FOCUS_LAYOUT_ORIGINAL walks tiles in token
+ *               order and skips dead far tiles; FOCUS_LAYOUT_CLASS_SORTED gathers Q/K/V into the
+ *               class-sorted order kept in the workspace, walks only sharing class pairs plus the
+ *               window, and scatters O/lse back to token order.
+ *   lse         device fp32 [batch*Hq, n], natural log
+ *   dev_status  device int32[4], nullable: [0] is set non-zero if a bounded wait inside the kernel
+ *               expired (the kernel then drains and exits; outputs are invalid), [1..3] say where.
+ *               The caller zeroes it and reads it after synchronising.
+ */
+FOCUS_API int focus_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k, focus_tensor v,
+                   const uint32_t* mq, const uint32_t* mk, const void* tiles_ws, int32_t layout,
+                   focus_tensor o, float* lse, int32_t* dev_status, void* stream);
+
+/*
+ * focus_count_kept -- exact number of attended pairs per query head (the denominator-free
+ * numerator of "effective FLOP": 4*D flop per attended pair).  Uses the gbits summaries of a
+ * workspace built for the same shape and masks (either layout).
+ *   counts_out  device uint64 [batch*Hq]; overwritten.
+ */
+FOCUS_API int focus_count_kept(const focus_shape* shape, const uint32_t* mq, const void* tiles_ws,
+                     unsigned long long* counts_out, void* stream);
+
+/*
+ * focus_selftest_umma -- diagnostic, not on the hot path (the paper has no counterpart): one
+ * 128 x 128 x D tile S = A B^T and one 128 x D x 128 tile O = P V through the same TMA, descriptor
+ * and tcgen05 building blocks as focus_attn_fwd, so that an encoding mistake shows up in isolation.
+ *   a, b, v   device bf16 [128, D] row-major     p   device bf16 [128, 128] row-major
+ *   s_out     device fp32 [128, 128]             o_out   device fp32 [128, D]
+ *   dev_status device int32, zeroed by the caller; non-zero if a bounded wait expired
+ */
+FOCUS_API int focus_selftest_umma(int32_t D, const void* a, const void* b, const void* p, const void* v, float* s_out,
+                        float* o_out, int32_t* dev_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FOCUS_H_ */

@@ -1,0 +1,206 @@
+// C-ABI entry points: argument validation, workspace layout, dispatch.  No kernels here.
+#include "common.cuh"
+
+#include <stdlib.h>
+#include <string.h>
+
+namespace focus {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+}
+
+int fail(int status, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+    return status;
+}
+
+int check_cuda(cudaError_t e, const char* what) {
+    if (e == cudaSuccess) return FOCUS_OK;
+    return fail(FOCUS_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+int validate_shape(const focus_shape* s) {
+    if (!s) return fail(FOCUS_ERR_INVALID_ARG, "shape is NULL");
+    if (s->batch < 1 || s->Hq < 1 || s->Hkv < 1 || s->n < 1)
+        return fail(FOCUS_ERR_INVALID_ARG, "batch, Hq, Hkv and n must be >= 1");
+    if (s->Hq % s->Hkv) return fail(FOCUS_ERR_INVALID_ARG, "Hq (%d) is not a multiple of Hkv (%d)", s->Hq, s->Hkv);
+    if (s->K < 1 || s->K > 32) return fail(FOCUS_ERR_INVALID_ARG, "K (%d) outside [1,32]", s->K);
+    if (s->topk < 1 || s->topk > s->K) return fail(FOCUS_ERR_INVALID_ARG, "topk (%d) outside [1,K]", s->topk);
+    if (s->window < 0) return fail(FOCUS_ERR_INVALID_ARG, "window must be >= 0");
+    if (!(s->scale >= 0.f) || !(s->softcap >= 0.f))
+        return fail(FOCUS_ERR_INVALID_ARG, "scale and softcap must be >= 0 (0 = default / off)");
+    if (s->D != 64 && s->D != 128 && s->D != 256)
+        return fail(FOCUS_ERR_UNSUPPORTED, "D (%d) must be 64, 128 or 256", s->D);
+    if ((long long)s->batch * s->Hq > (1 << 20)) return fail(FOCUS_ERR_INVALID_ARG, "batch*Hq too large");
+    if (s->n > (1 << 30)) return fail(FOCUS_ERR_INVALID_ARG, "n too large");
+    return FOCUS_OK;
+}
+
+int validate_tensor(const char* name, const focus_tensor& t, bool tma) {
+    if (!t.ptr) return fail(FOCUS_ERR_INVALID_ARG, "%s.ptr is NULL", name);
+    if (t.stride_n < 1 || t.stride_h < 1 || t.stride_b < 0)
+        return fail(FOCUS_ERR_INVALID_ARG, "%s has a non-positive stride", name);
+    if (tma) {
+        if ((uintptr_t)t.ptr % 16) return fail(FOCUS_ERR_INVALID_ARG, "%s.ptr is not 16-byte aligned", name);
+        if (t.stride_n % 8 || t.stride_h % 8 || t.stride_b % 8)
+            return fail(FOCUS_ERR_INVALID_ARG, "%s strides must be multiples of 8 elements", name);
+    }
+    return FOCUS_OK;
+}
+
+int require_sm100() {
+    int dev = 0, major = 0;
+    int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
+    if (rc) return rc;
+    rc = check_cuda(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev), "cudaDeviceGetAttribute");
+    if (rc) return rc;
+    if (major != 10) return fail(FOCUS_ERR_ARCH, "device compute capability %d.x is not 10.x (B200)", major);
+    return FOCUS_OK;
+}
+
+static int layout_of(const focus_shape* s, int layout, focus_tiles_layout* L) {
+    int rc = validate_shape(s);
+    if (rc) return rc;
+    if (!L) return fail(FOCUS_ERR_INVALID_ARG, "out is NULL");
+    if (layout != FOCUS_LAYOUT_ORIGINAL && layout != FOCUS_LAYOUT_CLASS_SORTED)
+        return fail(FOCUS_ERR_INVALID_ARG, "layout must be 0 (original) or 1 (class-sorted)");
+    memset(L, 0, sizeof *L);
+    const size_t HQ = (size_t)s->batch * s->Hq, HK = (size_t)s->batch * s->Hkv;
+    L->layout = layout;
+    L->nqt = cdiv(s->n, FOCUS_TILE_M);
+    L->nkt = cdiv(s->n, FOCUS_TILE_N);
+    L->nkw = cdiv(L->nkt, 32);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L->counters = take(8 * sizeof(uint64_t));
+    L->orq = take(HQ * L->nqt * 4);
+    L->andq = take(HQ * L->nqt * 4);
+    L->ork = take(HK * L->nkt * 4);
+    L->andk = take(HK * L->nkt * 4);
+    L->gbits = take(HK * L->nkt * (size_t)s->K * 4 * 4);
+    L->live = take(HQ * L->nqt * (size_t)L->nkw * 4);
+    L->live_cnt = take(HQ * L->nqt * 4);
+    if (layout == FOCUS_LAYOUT_CLASS_SORTED) {
+        L->nqp = sorted_capacity(s->n);
+        L->nkp = sorted_capacity(s->n);
+        L->ncls_q = take(HQ * 4);
+        L->ncls_k = take(HK * 4);
+        L->cls_q = take(HQ * FOCUS_MAX_CLASSES * 4);
+        L->cls_k = take(HK * FOCUS_MAX_CLASSES * 4);
+        L->seg_q = take(HQ * (FOCUS_MAX_CLASSES + 1) * 4);
+        L->seg_k = take(HK * (FOCUS_MAX_CLASSES + 1) * 4);
+        L->perm_q = take(HQ * (size_t)L->nqp * 4);
+        L->perm_k = take(HK * (size_t)L->nkp * 4);
+        L->qrange = take(HQ * (size_t)(L->nqp / 256) * FOCUS_MAX_CLASSES * 2 * 4);
+        L->qs = take(HQ * (size_t)L->nqp * s->D * 2);
+        L->ks = take(HK * (size_t)L->nkp * s->D * 2);
+        L->vs = take(HK * (size_t)L->nkp * s->D * 2);
+    }
+    L->total_bytes = off;
+    return FOCUS_OK;
+}
+
+}  // namespace focus
+
+using namespace focus;
+
+extern "C" {
+
+int focus_version(void) { return 100; }
+
+const char* focus_status_string(int status) {
+    switch (status) {
+        case FOCUS_OK: return "ok";
+        case FOCUS_ERR_INVALID_ARG: return "invalid argument";
+        case FOCUS_ERR_UNSUPPORTED: return "unsupported configuration";
+        case FOCUS_ERR_CAPACITY: return "workspace too small";
+        case FOCUS_ERR_ARCH: return "device is not sm_100";
+        case FOCUS_ERR_CUDA: return "CUDA error";
+        default: return "unknown status";
+    }
+}
+
+const char* focus_last_error(void) { return g_err; }
+
+int focus_tiles_layout_of(const focus_shape* shape, int32_t layout, focus_tiles_layout* out) {
+    return layout_of(shape, layout, out);
+}
+
+size_t focus_tiles_workspace_bytes(const focus_shape* shape, int32_t layout) {
+    focus_tiles_layout L;
+    if (layout_of(shape, layout, &L)) return 0;
+    return L.total_bytes;
+}
+
+int focus_assign(const focus_shape* shape, focus_tensor x, int32_t H, const float* centroids, uint32_t* masks_out,
+                 unsigned long long* near_ties, float near_tie_eps, void* stream) {
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if (H != shape->Hq && H != shape->Hkv) return fail(FOCUS_ERR_INVALID_ARG, "H (%d) must be Hq or Hkv", H);
+    if ((rc = validate_tensor("x", x, false))) return rc;
+    if ((uintptr_t)x.ptr % 16 || x.stride_n % 8 || x.stride_h % 8 || x.stride_b % 8)
+        return fail(FOCUS_ERR_INVALID_ARG, "x must be 16-byte aligned with strides that are multiples of 8 elements");
+    if (!centroids || !masks_out) return fail(FOCUS_ERR_INVALID_ARG, "centroids or masks_out is NULL");
+    if ((rc = require_sm100())) return rc;
+    return launch_assign(shape, x, H, centroids, masks_out, near_ties, near_tie_eps, (cudaStream_t)stream);
+}
+
+int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, const uint32_t* mk, int32_t layout, void* ws,
+                      size_t ws_bytes, void* stream) {
+    focus_tiles_layout L;
+    int rc = layout_of(shape, layout, &L);
+    if (rc) return rc;
+    if (!mq || !mk || !ws) return fail(FOCUS_ERR_INVALID_ARG, "mq, mk or ws is NULL");
+    if ((uintptr_t)ws % 256) return fail(FOCUS_ERR_INVALID_ARG, "ws is not 256-byte aligned");
+    if (ws_bytes < L.total_bytes)
+        return fail(FOCUS_ERR_CAPACITY, "workspace has %zu bytes, %zu needed", ws_bytes, L.total_bytes);
+    if ((rc = require_sm100())) return rc;
+    return launch_build_tiles(shape, mq, mk, layout, L, (char*)ws, (cudaStream_t)stream);
+}
+
+int focus_count_kept(const focus_shape* shape, const uint32_t* mq, const void* tiles_ws,
+                     unsigned long long* counts_out, void* stream) {
+    focus_tiles_layout L;
+    int rc = layout_of(shape, FOCUS_LAYOUT_ORIGINAL, &L);   // the summaries sit at the same offsets in both layouts
+    if (rc) return rc;
+    if (!mq || !tiles_ws || !counts_out) return fail(FOCUS_ERR_INVALID_ARG, "mq, tiles_ws or counts_out is NULL");
+    if ((rc = require_sm100())) return rc;
+    return launch_count_kept(shape, mq, L, (const char*)tiles_ws, counts_out, (cudaStream_t)stream);
+}
+
+int focus_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k, focus_tensor v, const uint32_t* mq,
+                   const uint32_t* mk, const void* tiles_ws, int32_t layout, focus_tensor o, float* lse,
+                   int32_t* dev_status, void* stream) {
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if ((rc = validate_tensor("q", q, true)) || (rc = validate_tensor("k", k, true)) ||
+        (rc = validate_tensor("v", v, true)) || (rc = validate_tensor("o", o, true)))
+        return rc;
+    if (!lse) return fail(FOCUS_ERR_INVALID_ARG, "lse is NULL");
+    if (tiles_ws && (!mq || !mk)) return fail(FOCUS_ERR_INVALID_ARG, "mq/mk are required with a tiles workspace");
+    if ((rc = require_sm100())) return rc;
+    AttnArgs a;
+    a.s = *shape;
+    a.q = q; a.k = k; a.v = v; a.o = o;
+    a.mq = mq; a.mk = mk;
+    a.ws = (const char*)tiles_ws;
+    a.lse = lse;
+    a.dev_status = dev_status;
+    a.scale = shape->scale > 0.f ? shape->scale : 1.0f / sqrtf((float)shape->D);
+    memset(&a.L, 0, sizeof a.L);
+    if (tiles_ws && (rc = layout_of(shape, layout, &a.L))) return rc;
+    const char* impl = getenv("FOCUS_ATTN_IMPL");
+    if (impl && !strcmp(impl, "simple")) return launch_attn_simple(a, (cudaStream_t)stream);
+    return launch_attn_sm100(a, (cudaStream_t)stream);
+}
+
+}  // extern "C"

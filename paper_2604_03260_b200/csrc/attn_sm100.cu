@@ -1,0 +1,528 @@
+// focus_attn_fwd for sm_100a: persistent, warp-specialised attention forward over the attended
+// pairs of the Focus mask (paper Sec. 2 and Appendix C, first equation).
+//
+// One CTA per SM works through (head, 256-query block) items.  Per item, two 128-row query tiles
+// share every key/value tile that is fetched:
+//   warp 0        TMA producer: Q tiles once per item, then K and V tiles of every visited key tile
+//                 into a ring of shared-memory stages (128-byte swizzle)
+//   warp 1        MMA issuer: S_x = Q_x K^T and O_x += P_x V with tcgen05.mma, accumulators in TMEM
+//   warps 4-7     softmax for query tile 0: tcgen05.ld S, mask, online max/sum, P (bf16) back to TMEM
+//   warps 8-11    softmax for query tile 1
+// The two softmax groups alternate on the tensor pipe: while one computes exponentials the MMAs of
+// the other run.  The running maximum is raised lazily (only when it grows by more than 2^8), and
+// then the owner of the row rescales its O row in TMEM itself.
+//
+// Which key tiles are visited: in dense mode every tile up to the diagonal; with a tiles
+// workspace, far tiles (every pair beyond the window) only when the live bitmap says the OR of the
+// query-tile masks meets the OR of the key-tile masks; near tiles always.
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+#include "tma_host.cuh"
+
+namespace focus {
+
+using namespace ptx;
+
+constexpr int ATT_THREADS = 384;
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr float LN2 = 0.6931471805599453f;
+constexpr float RESCALE_THRESHOLD = 8.0f;   // log2 units: the stale maximum may lag by a factor of 256
+
+struct AttnParams {
+    int B, Hq, Hkv, G, n, w, K;
+    int nqb;                 // 256-row query blocks per head
+    int nqt, nkt, nkw;
+    int dense;
+    float scale, softcap;
+    const uint32_t* mq;
+    const uint32_t* gbits;
+    const uint32_t* live;
+    const uint32_t* andq;
+    const uint32_t* andk;
+    __nv_bfloat16* o;
+    int64_t o_sb, o_sh, o_sn;
+    float* lse;
+    int32_t* status;
+    long long nitems;
+};
+
+// Enumerates the key tiles a 256-row query block visits, in increasing order.  Every role of the
+// CTA runs the same walk over the same data, which keeps them in step without communication.
+struct TileWalk {
+    const uint32_t* l0;
+    const uint32_t* l1;
+    int f0, b_last, b, wd;
+    uint32_t bits;
+    bool far_phase;
+
+    __device__ __forceinline__ void init(const AttnParams& p, int hq, int A) {
+        const int a0 = 2 * A;
+        const long long last_row = min((long long)p.n, (long long)(A + 1) * 256) - 1;
+        b_last = (int)(last_row / 128);
+        f0 = 0;
+        l0 = l1 = nullptr;
+        if (!p.dense) {
+            const long long d = (long long)a0 * 128 - p.w;
+            f0 = d > 0 ? (int)(d / 128) : 0;
+            l0 = p.live + ((size_t)hq * p.nqt + a0) * p.nkw;
+            if (a0 + 1 < p.nqt) l1 = l0 + p.nkw;
+        }
+        far_phase = f0 > 0;
+        wd = -1;
+        bits = 0;
+        b = f0;
+    }
+    __device__ __forceinline__ int next() {
+        if (far_phase) {
+            for (;;) {
+                if (bits) {
+                    const int c = __ffs(bits) - 1;
+                    bits &= bits - 1;
+                    return wd * 32 + c;
+                }
+                ++wd;
+                if (wd * 32 >= f0) { far_phase = false; break; }
+                uint32_t x = __ldg(l0 + wd);
+                if (l1) x |= __ldg(l1 + wd);
+                const int rem = f0 - wd * 32;
+                if (rem < 32) x &= (1u << rem) - 1u;
+                bits = x;
+            }
+        }
+        if (b <= b_last) return b++;
+        return -1;
+    }
+};
+
+template <int D>
+struct AttnCfg {
+    static constexpr int SUBT = D / 64;
+    static constexpr uint32_t SUB_BYTES = 128 * 64 * 2;
+    static constexpr uint32_t TILE_BYTES = SUB_BYTES * SUBT;
+    static constexpr int NSTAGE = (D == 128) ? 5 : 8;
+    static constexpr uint32_t SMEM_BYTES = 1024 + 2 * TILE_BYTES + NSTAGE * TILE_BYTES;
+    static constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O0 = 256, COL_O1 = 256 + D;
+};
+
+struct SharedCtl {
+    uint64_t q_full, q_empty;
+    uint64_t s_full[2], p_full[2], o_full[2];
+    uint64_t kv_full[8], kv_empty[8];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+// bounded wait that also gives up when another role of the CTA has already given up
+__device__ __forceinline__ bool ctl_wait(uint64_t* bar, uint32_t parity, SharedCtl* ctl) {
+    const uint32_t a = smem_u32(bar);
+    if (mbar_try_wait(a, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int it = 0; it < 128; ++it)
+            if (mbar_try_wait(a, parity)) return true;
+        if (*(volatile int*)&ctl->abort_flag) return false;
+        if (globaltimer_ns() - t0 > 4000000000ull) return false;
+    }
+}
+
+__device__ __forceinline__ void report_timeout(const AttnParams& p, SharedCtl* ctl, int where, int item) {
+    *(volatile int*)&ctl->abort_flag = 1;
+    if (p.status && atomicCAS(p.status, 0, 1) == 0) {
+        p.status[1] = where;
+        p.status[2] = item;
+        p.status[3] = (int)blockIdx.x;
+    }
+}
+
+template <int D, bool SOFTCAP>
+__global__ void __launch_bounds__(ATT_THREADS, 1)
+focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                  const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
+    using C = AttnCfg<D>;
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ __align__(8) SharedCtl ctl;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sq = base;                                // 2 query tiles
+    const uint32_t skv = base + 2 * C::TILE_BYTES;            // ring of K / V tiles
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int HQ = p.B * p.Hq;
+
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&ctl.q_full), 1);
+        mbar_init(smem_u32(&ctl.q_empty), 1);
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(smem_u32(&ctl.s_full[x]), 1);
+            mbar_init(smem_u32(&ctl.p_full[x]), 128);
+            mbar_init(smem_u32(&ctl.o_full[x]), 1);
+        }
+        for (int s = 0; s < C::NSTAGE; ++s) {
+            mbar_init(smem_u32(&ctl.kv_full[s]), 1);
+            mbar_init(smem_u32(&ctl.kv_empty[s]), 1);
+        }
+        ctl.abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&ctl.tmem_base), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = ctl.tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
+            long long nload = 0;
+            int it = 0;
+            bool ok = true;
+            for (long long item = blockIdx.x; ok && item < p.nitems; item += gridDim.x, ++it) {
+                const int A = p.nqb - 1 - (int)(item / HQ);
+                const int hq = (int)(item % HQ);
+                const int b = hq / p.Hq, h = hq % p.Hq, hk = h / p.G;
+                if (it > 0 && !ctl_wait(&ctl.q_empty, (it - 1) & 1, &ctl)) { report_timeout(p, &ctl, 10, (int)item); break; }
+                mbar_arrive_expect_tx(smem_u32(&ctl.q_full), 2 * C::TILE_BYTES);
+                for (int x = 0; x < 2; ++x)
+                    for (int c = 0; c < C::SUBT; ++c)
+                        tma_load_4d(sq + x * C::TILE_BYTES + c * C::SUB_BYTES, &tm_q, smem_u32(&ctl.q_full), c * 64,
+                                    A * 256 + x * 128, h, b);
+                TileWalk walk;
+                walk.init(p, hq, A);
+                int kb;
+                while (ok && (kb = walk.next()) >= 0) {
+                    for (int kv = 0; kv < 2; ++kv) {
+                        const int slot = (int)(nload % C::NSTAGE);
+                        const long long use = nload / C::NSTAGE;
+                        if (use > 0 && !ctl_wait(&ctl.kv_empty[slot], (uint32_t)((use - 1) & 1), &ctl)) {
+                            report_timeout(p, &ctl, 11, (int)item);
+                            ok = false;
+                            break;
+                        }
+                        const uint32_t bar = smem_u32(&ctl.kv_full[slot]);
+                        mbar_arrive_expect_tx(bar, C::TILE_BYTES);
+                        for (int c = 0; c < C::SUBT; ++c)
+                            tma_load_4d(skv + slot * C::TILE_BYTES + c * C::SUB_BYTES, kv ? &tm_v : &tm_k, bar, c * 64,
+                                        kb * 128, hk, b);
+                        ++nload;
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t IDESC_S = idesc_bf16(128, 128, 0, 0);
+            constexpr uint32_t IDESC_O = idesc_bf16(128, D, 0, 1);
+            long long nuse = 0;             // K/V stages consumed so far
+            uint32_t np[2] = {0, 0};        // P tiles consumed per query tile
+            int it = 0;
+            bool ok = true;
+            auto issue_s = [&](int x, uint32_t kaddr) {
+                const uint32_t d = tmem + (x ? C::COL_S1 : C::COL_S0);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off = (ks / 4) * C::SUB_BYTES + (ks % 4) * 32;
+                    umma_ss(d, smem_desc_sw128(sq + x * C::TILE_BYTES + off, 16, 1024),
+                            smem_desc_sw128(kaddr + off, 16, 1024), IDESC_S, ks > 0);
+                }
+            };
+            auto issue_o = [&](int x, uint32_t vaddr, bool first) {
+                const uint32_t d = tmem + (x ? C::COL_O1 : C::COL_O0);
+                const uint32_t a = tmem + (x ? C::COL_S1 : C::COL_S0);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    umma_ts(d, a + ks * 8, smem_desc_sw128(vaddr + ks * 2048, C::SUB_BYTES, 1024), IDESC_O,
+                            (!first) || ks > 0);
+            };
+            for (long long item = blockIdx.x; ok && item < p.nitems; item += gridDim.x, ++it) {
+                const int A = p.nqb - 1 - (int)(item / HQ);
+                const int hq = (int)(item % HQ);
+                TileWalk walk;
+                walk.init(p, hq, A);
+                int cur = walk.next();
+                if (!ctl_wait(&ctl.q_full, it & 1, &ctl)) { report_timeout(p, &ctl, 20, (int)item); break; }
+                // S of the first tile for both query tiles
+                {
+                    const int slot = (int)(nuse % C::NSTAGE);
+                    if (!ctl_wait(&ctl.kv_full[slot], (uint32_t)((nuse / C::NSTAGE) & 1), &ctl)) {
+                        report_timeout(p, &ctl, 21, (int)item); break;
+                    }
+                    tc_fence_after();
+                    const uint32_t kaddr = skv + slot * C::TILE_BYTES;
+                    issue_s(0, kaddr); umma_commit(smem_u32(&ctl.s_full[0]));
+                    issue_s(1, kaddr); umma_commit(smem_u32(&ctl.s_full[1]));
+                    umma_commit(smem_u32(&ctl.kv_empty[slot]));
+                    ++nuse;
+                }
+                bool first = true;
+                while (cur >= 0) {
+                    const int nxt = walk.next();
+                    const int vslot = (int)(nuse % C::NSTAGE);
+                    if (!ctl_wait(&ctl.kv_full[vslot], (uint32_t)((nuse / C::NSTAGE) & 1), &ctl)) {
+                        report_timeout(p, &ctl, 22, (int)item); ok = false; break;
+                    }
+                    ++nuse;
+                    const uint32_t vaddr = skv + vslot * C::TILE_BYTES;
+                    int kslot = 0;
+                    uint32_t kaddr = 0;
+                    if (nxt >= 0) {
+                        kslot = (int)(nuse % C::NSTAGE);
+                        if (!ctl_wait(&ctl.kv_full[kslot], (uint32_t)((nuse / C::NSTAGE) & 1), &ctl)) {
+                            report_timeout(p, &ctl, 23, (int)item); ok = false; break;
+                        }
+                        ++nuse;
+                        kaddr = skv + kslot * C::TILE_BYTES;
+                    } else {
+                        umma_commit(smem_u32(&ctl.q_empty));     // every S of this item has been issued
+                    }
+                    // query tile 0
+                    if (!ctl_wait(&ctl.p_full[0], np[0] & 1, &ctl)) { report_timeout(p, &ctl, 24, (int)item); ok = false; break; }
+                    ++np[0];
+                    tc_fence_after();
+                    issue_o(0, vaddr, first);
+                    if (nxt >= 0) { issue_s(0, kaddr); umma_commit(smem_u32(&ctl.s_full[0])); }
+                    else umma_commit(smem_u32(&ctl.o_full[0]));
+                    // query tile 1
+                    if (!ctl_wait(&ctl.p_full[1], np[1] & 1, &ctl)) { report_timeout(p, &ctl, 25, (int)item); ok = false; break; }
+                    ++np[1];
+                    tc_fence_after();
+                    issue_o(1, vaddr, first);
+                    umma_commit(smem_u32(&ctl.kv_empty[vslot]));
+                    if (nxt >= 0) {
+                        issue_s(1, kaddr); umma_commit(smem_u32(&ctl.s_full[1]));
+                        umma_commit(smem_u32(&ctl.kv_empty[kslot]));
+                    } else {
+                        umma_commit(smem_u32(&ctl.o_full[1]));
+                    }
+                    first = false;
+                    cur = nxt;
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------------ softmax + epilogue
+        const int x = (warp - 4) >> 2;                       // query tile of this warpgroup
+        const int row_in_tile = ((warp & 3) << 5) | lane;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t t_s = tmem + lane_base + (x ? C::COL_S1 : C::COL_S0);
+        const uint32_t t_o = tmem + lane_base + (x ? C::COL_O1 : C::COL_O0);
+        const float sl2 = SOFTCAP ? LOG2E : p.scale * LOG2E;
+        const float cap_in = SOFTCAP ? p.scale / p.softcap : 0.f;
+        uint32_t ns = 0;
+        int it = 0;
+        bool ok = true;
+        for (long long item = blockIdx.x; ok && item < p.nitems; item += gridDim.x, ++it) {
+            const int A = p.nqb - 1 - (int)(item / HQ);
+            const int hq = (int)(item % HQ);
+            const int bb = hq / p.Hq, h = hq % p.Hq;
+            const int hk = bb * p.Hkv + h / p.G;
+            const int a = 2 * A + x;
+            const long long i = (long long)a * 128 + row_in_tile;
+            const bool valid = i < p.n;
+            const uint32_t mi = (valid && !p.dense) ? __ldg(p.mq + (size_t)hq * p.n + i) : 0u;
+            const uint32_t aq = (!p.dense && a < p.nqt) ? __ldg(p.andq + (size_t)hq * p.nqt + a) : 0u;
+            const long long dfar = (long long)a * 128 - p.w;
+            const int f_x = (!p.dense && dfar > 0) ? (int)(dfar / 128) : 0;   // tiles b < f_x are far for this query tile
+            const long long r_last = (long long)a * 128 + 127;
+            float m_used = -INFINITY, l = 0.f;
+            TileWalk walk;
+            walk.init(p, hq, A);
+            int kb;
+            bool first = true;
+            while ((kb = walk.next()) >= 0) {
+                const long long c0 = (long long)kb * 128;
+                // ---- how this tile is masked for this query tile (uniform over the warpgroup)
+                bool all_masked = c0 > r_last || (long long)a * 128 >= p.n;
+                bool need_causal = c0 + 127 > (long long)a * 128;
+                bool need_group = false, need_window = false;
+                if (!p.dense && !all_masked) {
+                    if (kb < f_x) {
+                        need_group = !(aq & __ldg(p.andk + (size_t)hk * p.nkt + kb));
+                    } else if (r_last - c0 > p.w) {
+                        need_group = need_window = true;
+                    }
+                }
+                uint32_t kw[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
+                const bool masked = need_causal || need_group;
+                if (masked && !all_masked) {
+                    uint32_t sh[4] = {0, 0, 0, 0};
+                    if (need_group) {
+                        const uint32_t* gb = p.gbits + ((size_t)hk * p.nkt + kb) * p.K * 4;
+                        uint32_t rem = mi;
+                        while (rem) {
+                            const int g = __ffs(rem) - 1;
+                            rem &= rem - 1;
+                            if (g < p.K) {
+                                const uint4 t = __ldg(reinterpret_cast<const uint4*>(gb + g * 4));
+                                sh[0] |= t.x; sh[1] |= t.y; sh[2] |= t.z; sh[3] |= t.w;
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t keep = 0xffffffffu;
+                        if (need_group) {
+                            keep = sh[q];
+                            if (need_window) {
+                                const long long lo = i - p.w - c0 - 32 * q;      // columns >= lo are inside the window
+                                keep |= lo <= 0 ? 0xffffffffu : (lo >= 32 ? 0u : ~((1u << (int)lo) - 1u));
+                            }
+                        }
+                        if (need_causal) {
+                            const long long nk = i - c0 + 1 - 32 * q;            // columns < nk are causal
+                            keep &= nk >= 32 ? 0xffffffffu : (nk <= 0 ? 0u : ((1u << (int)nk) - 1u));
+                        }
+                        kw[q] = keep;
+                    }
+                }
+                // ---- wait for S
+                if (!ctl_wait(&ctl.s_full[x], ns & 1, &ctl)) { report_timeout(p, &ctl, 30 + x, (int)item); ok = false; break; }
+                ++ns;
+                tc_fence_after();
+                uint32_t pk[64];
+                if (all_masked) {
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) pk[c] = 0u;
+                } else {
+                    uint32_t sr[128];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) tmem_ld32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[c * 32]));
+                    tmem_wait_ld();
+                    float mt = -INFINITY;
+#pragma unroll
+                    for (int c = 0; c < 128; ++c) {
+                        float s = __uint_as_float(sr[c]);
+                        if (SOFTCAP) s = p.softcap * tanh_approx(s * cap_in);
+                        if (masked) s = ((kw[c >> 5] >> (c & 31)) & 1u) ? s : -INFINITY;
+                        sr[c] = __float_as_uint(s);
+                        mt = fmaxf(mt, s);
+                    }
+                    mt *= sl2;                                      // log2 units (sl2 > 0; -inf stays -inf)
+                    // ---- lazy maximum: raise the reference only when it lags by more than the threshold
+                    float factor = 1.f;
+                    bool raise = false;
+                    if (m_used == -INFINITY) {
+                        m_used = mt;                                 // nothing accumulated yet for this row
+                    } else if (mt > m_used + RESCALE_THRESHOLD) {
+                        factor = ex2_approx(m_used - mt);
+                        m_used = mt;
+                        raise = true;
+                    }
+                    if (__any_sync(0xffffffffu, raise) && !first) {
+                        // the previous PV of this query tile has completed (its commit precedes s_full)
+#pragma unroll 1
+                        for (int c = 0; c < D / 16; ++c) {
+                            uint32_t ov[16];
+                            tmem_ld16(t_o + c * 16, ov);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * factor);
+                            tmem_st16(t_o + c * 16, ov);
+                        }
+                    }
+                    l *= factor;
+                    const float msub = m_used == -INFINITY ? 0.f : m_used;
+                    float rs0 = 0.f, rs1 = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 128; c += 2) {
+                        const float p0 = ex2_approx(fmaf(__uint_as_float(sr[c]), sl2, -msub));
+                        const float p1 = ex2_approx(fmaf(__uint_as_float(sr[c + 1]), sl2, -msub));
+                        rs0 += p0;
+                        rs1 += p1;
+                        pk[c >> 1] = pack_bf16x2(p0, p1);
+                    }
+                    l += rs0 + rs1;
+                }
+                tmem_st32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+                tmem_st32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(smem_u32(&ctl.p_full[x]));
+                first = false;
+            }
+            if (!ok) break;
+            // ---- epilogue: O / l -> bf16 -> global, lse
+            if (!ctl_wait(&ctl.o_full[x], it & 1, &ctl)) { report_timeout(p, &ctl, 40 + x, (int)item); break; }
+            tc_fence_after();
+            const float inv_l = 1.f / l;
+            __nv_bfloat16* orow = p.o + (size_t)bb * p.o_sb + (size_t)h * p.o_sh + (size_t)(valid ? i : 0) * p.o_sn;
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t ov[32];
+                tmem_ld32(t_o + c * 32, ov);
+                tmem_wait_ld();
+                if (valid) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8) {
+                        uint4 w4;
+                        w4.x = pack_bf16x2(__uint_as_float(ov[e]) * inv_l, __uint_as_float(ov[e + 1]) * inv_l);
+                        w4.y = pack_bf16x2(__uint_as_float(ov[e + 2]) * inv_l, __uint_as_float(ov[e + 3]) * inv_l);
+                        w4.z = pack_bf16x2(__uint_as_float(ov[e + 4]) * inv_l, __uint_as_float(ov[e + 5]) * inv_l);
+                        w4.w = pack_bf16x2(__uint_as_float(ov[e + 6]) * inv_l, __uint_as_float(ov[e + 7]) * inv_l);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + e) = w4;
+                    }
+                }
+            }
+            if (valid) p.lse[(size_t)hq * p.n + i] = (m_used + lg2_approx(l)) * LN2;
+            tc_fence_before();
+        }
+    }
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+template <int D, bool SOFTCAP>
+static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
+    using C = AttnCfg<D>;
+    CUtensorMap tq, tk, tv;
+    int rc;
+    if ((rc = make_tmap_qkv(&tq, a.q, a.s.batch, a.s.Hq, a.s.n, D))) return rc;
+    if ((rc = make_tmap_qkv(&tk, a.k, a.s.batch, a.s.Hkv, a.s.n, D))) return rc;
+    if ((rc = make_tmap_qkv(&tv, a.v, a.s.batch, a.s.Hkv, a.s.n, D))) return rc;
+    AttnParams p;
+    p.B = a.s.batch; p.Hq = a.s.Hq; p.Hkv = a.s.Hkv; p.G = a.s.Hq / a.s.Hkv; p.n = a.s.n; p.w = a.s.window; p.K = a.s.K;
+    p.nqb = cdiv(a.s.n, 256);
+    p.nqt = cdiv(a.s.n, 128); p.nkt = cdiv(a.s.n, 128); p.nkw = cdiv(p.nkt, 32);
+    p.dense = a.ws ? 0 : 1;
+    p.scale = a.scale; p.softcap = a.s.softcap;
+    p.mq = a.mq;
+    p.gbits = a.ws ? reinterpret_cast<const uint32_t*>(a.ws + a.L.gbits) : nullptr;
+    p.live = a.ws ? reinterpret_cast<const uint32_t*>(a.ws + a.L.live) : nullptr;
+    p.andq = a.ws ? reinterpret_cast<const uint32_t*>(a.ws + a.L.andq) : nullptr;
+    p.andk = a.ws ? reinterpret_cast<const uint32_t*>(a.ws + a.L.andk) : nullptr;
+    p.o = reinterpret_cast<__nv_bfloat16*>(a.o.ptr);
+    p.o_sb = a.o.stride_b; p.o_sh = a.o.stride_h; p.o_sn = a.o.stride_n;
+    p.lse = a.lse;
+    p.status = a.dev_status;
+    p.nitems = (long long)a.s.batch * a.s.Hq * p.nqb;
+    int dev = 0, sms = 0;
+    if ((rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice"))) return rc;
+    if ((rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "cudaDeviceGetAttribute"))) return rc;
+    auto kern = focus_attn_kernel<D, SOFTCAP>;
+    if ((rc = check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES),
+                         "cudaFuncSetAttribute(attn)")))
+        return rc;
+    const int grid = (int)(p.nitems < sms ? p.nitems : sms);
+    kern<<<grid, ATT_THREADS, C::SMEM_BYTES, st>>>(tq, tk, tv, p);
+    return check_cuda(cudaGetLastError(), "attention kernel launch");
+}
+
+int launch_attn_sm100(const AttnArgs& a, cudaStream_t st) {
+    if (a.ws && a.L.layout == FOCUS_LAYOUT_CLASS_SORTED)
+        return fail(FOCUS_ERR_UNSUPPORTED, "class-sorted layout is not available in the tensor-core kernel yet");
+    const bool cap = a.s.softcap > 0.f;
+    switch (a.s.D) {
+        case 64: return cap ? launch_attn_t<64, true>(a, st) : launch_attn_t<64, false>(a, st);
+        case 128: return cap ? launch_attn_t<128, true>(a, st) : launch_attn_t<128, false>(a, st);
+    }
+    return fail(FOCUS_ERR_UNSUPPORTED, "head dimension %d is not available in the tensor-core kernel yet", a.s.D);
+}
+
+}  // namespace focus

@@ -1,0 +1,54 @@
+// Internal helpers shared by the translation units of libfocus_b200.so.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <stdarg.h>
+
+#include "focus.h"
+
+namespace focus {
+
+// thread-local error text behind focus_last_error()
+void set_error(const char* fmt, ...);
+int fail(int status, const char* fmt, ...);
+int check_cuda(cudaError_t e, const char* what);
+
+// shape validation shared by all entry points (0 or a negative status)
+int validate_shape(const focus_shape* s);
+// validation of a bf16 tensor argument; tma = also enforce 16-byte base alignment and stride % 8 == 0
+int validate_tensor(const char* name, const focus_tensor& t, bool tma);
+// current device must be compute capability 10.x
+int require_sm100();
+
+inline int cdiv(int a, int b) { return (a + b - 1) / b; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// layout-1 padded sorted length: room for every class segment to be rounded up to 256 slots
+inline int sorted_capacity(int n) { return (int)align_up((size_t)n + (size_t)FOCUS_MAX_CLASSES * 255, 256); }
+
+// launchers implemented in the other translation units
+int launch_assign(const focus_shape* s, const focus_tensor& x, int H, const float* centroids, uint32_t* masks,
+                  unsigned long long* near_ties, float eps, cudaStream_t st);
+int launch_build_tiles(const focus_shape* s, const uint32_t* mq, const uint32_t* mk, int layout,
+                       const focus_tiles_layout& L, char* ws, cudaStream_t st);
+int launch_count_kept(const focus_shape* s, const uint32_t* mq, const focus_tiles_layout& L, const char* ws,
+                      unsigned long long* out, cudaStream_t st);
+
+struct AttnArgs {
+    focus_shape s;
+    focus_tensor q, k, v, o;
+    const uint32_t* mq;
+    const uint32_t* mk;
+    const char* ws;           // nullptr = dense causal
+    focus_tiles_layout L;     // valid when ws != nullptr
+    float* lse;
+    int32_t* dev_status;
+    float scale;              // resolved logit scale
+};
+int launch_attn_simple(const AttnArgs& a, cudaStream_t st);
+int launch_attn_sm100(const AttnArgs& a, cudaStream_t st);
+
+}  // namespace focus

@@ -1,0 +1,99 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every symbol the header declares, and its
+host-only logic (validation, workspace layout) behaves.  No compute call is made here."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2604_03260_b200 import binding as fb
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "focus.h")).read()
+    return sorted(set(re.findall(r"FOCUS_API[^;(]*?\b(focus_\w+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_symbols()
+    assert {"focus_assign", "focus_build_tiles", "focus_attn_fwd", "focus_count_kept", "focus_version",
+            "focus_tiles_layout_of", "focus_tiles_workspace_bytes", "focus_status_string",
+            "focus_last_error"} <= set(names)
+    L = ctypes.CDLL(fb.LIB_PATH)
+    for n in names:
+        assert hasattr(L, n), n
+    assert fb.focus_version() >= 100
+
+
+def test_status_strings():
+    L = fb.lib()
+    assert L.focus_status_string(0) == b"ok"
+    for code in (-1, -2, -3, -4, -5):
+        assert L.focus_status_string(code) not in (b"ok", b"unknown status")
+    assert L.focus_status_string(-99) == b"unknown status"
+
+
+def test_workspace_layout_is_consistent():
+    s = fb.make_shape(32, 8, 131072 + 5, 128, 4, 2, 2048)
+    for layout in (0, 1):
+        L = fb.focus_tiles_layout_of(s, layout)
+        assert L.layout == layout and L.nqt == 1025 and L.nkt == 1025 and L.nkw == 33
+        assert L.total_bytes == fb.focus_tiles_workspace_bytes(s, layout)
+        offs = [L.counters, L.orq, L.andq, L.ork, L.andk, L.gbits, L.live, L.live_cnt]
+        sizes = [64, 32 * 1025 * 4, 32 * 1025 * 4, 8 * 1025 * 4, 8 * 1025 * 4, 8 * 1025 * 4 * 16, 32 * 1025 * 33 * 4,
+                 32 * 1025 * 4]
+        if layout == 1:
+            assert L.nqp % 256 == 0 and L.nqp >= s.n + 64 * 255
+            offs += [L.ncls_q, L.ncls_k, L.cls_q, L.cls_k, L.seg_q, L.seg_k, L.perm_q, L.perm_k, L.qrange, L.qs,
+                     L.ks, L.vs]
+            sizes += [32 * 4, 8 * 4, 32 * 64 * 4, 8 * 64 * 4, 32 * 65 * 4, 8 * 65 * 4, 32 * L.nqp * 4, 8 * L.nkp * 4,
+                      32 * (L.nqp // 256) * 64 * 8, 32 * L.nqp * 128 * 2, 8 * L.nkp * 128 * 2, 8 * L.nkp * 128 * 2]
+        for o, sz, nxt in zip(offs, sizes, offs[1:] + [L.total_bytes]):
+            assert o % 256 == 0 and o + sz <= nxt
+
+
+@pytest.mark.parametrize("kw,status", [
+    (dict(Hq=6, Hkv=4), -1), (dict(K=33), -1), (dict(K=0), -1), (dict(topk=5), -1), (dict(topk=0), -1),
+    (dict(window=-1), -1), (dict(n=0), -1), (dict(D=96), -2), (dict(batch=0), -1), (dict(scale=-1.0), -1),
+])
+def test_bad_shapes_are_rejected_on_the_host(kw, status):
+    base = dict(Hq=8, Hkv=4, n=1000, D=128, K=4, topk=2, window=16)
+    base.update(kw)
+    s = fb.make_shape(**base)
+    assert fb.focus_tiles_workspace_bytes(s, 0) == 0
+    out = fb.focus_tiles_layout()
+    assert fb.lib().focus_tiles_layout_of(ctypes.byref(s), 0, ctypes.byref(out)) == status
+    assert len(fb.lib().focus_last_error()) > 0
+
+
+def test_null_and_misaligned_arguments_never_reach_the_device():
+    s = fb.make_shape(8, 4, 1000, 128, 4, 2, 16)
+    L = fb.lib()
+    t_ok = fb.focus_tensor(4096, 8 * 1000 * 128, 1000 * 128, 128)
+    t_null = fb.focus_tensor(None, 1, 1, 1)
+    t_mis = fb.focus_tensor(4098, 8 * 1000 * 128, 1000 * 128, 128)
+    t_str = fb.focus_tensor(4096, 8 * 1000 * 132, 1000 * 132, 132)
+    assert L.focus_assign(ctypes.byref(s), t_null, 8, 4096, 4096, None, 1e-5, None) == -1
+    assert L.focus_assign(ctypes.byref(s), t_ok, 3, 4096, 4096, None, 1e-5, None) == -1
+    assert L.focus_assign(ctypes.byref(s), t_ok, 8, None, 4096, None, 1e-5, None) == -1
+    assert L.focus_build_tiles(ctypes.byref(s), None, 4096, 0, 4096, 1 << 30, None) == -1
+    assert L.focus_build_tiles(ctypes.byref(s), 4096, 4096, 0, 4096 + 8, 1 << 30, None) == -1     # ws alignment
+    assert L.focus_build_tiles(ctypes.byref(s), 4096, 4096, 0, 4096, 16, None) == -3               # capacity
+    assert L.focus_build_tiles(ctypes.byref(s), 4096, 4096, 7, 4096, 1 << 30, None) == -1          # layout id
+    for bad in (t_null, t_mis, t_str):
+        assert L.focus_attn_fwd(ctypes.byref(s), bad, t_ok, t_ok, None, None, None, 0, t_ok, 4096, None, None) == -1
+    assert L.focus_attn_fwd(ctypes.byref(s), t_ok, t_ok, t_ok, None, None, None, 0, t_ok, None, None, None) == -1
+    assert L.focus_attn_fwd(ctypes.byref(s), t_ok, t_ok, t_ok, None, None, 4096, 0, t_ok, 4096, None, None) == -1
+    assert L.focus_count_kept(ctypes.byref(s), None, 4096, 4096, None) == -1
+
+
+def test_without_a_device_the_library_reports_an_error_instead_of_computing():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    s = fb.make_shape(8, 4, 1000, 128, 4, 2, 16)
+    t_ok = fb.focus_tensor(4096, 8 * 1000 * 128, 1000 * 128, 128)
+    rc = fb.lib().focus_assign(ctypes.byref(s), t_ok, 8, 4096, 4096, None, 1e-5, None)
+    assert rc in (-4, -5)

@@ -1,0 +1,128 @@
+"""focus_attn_fwd vs the fp64 oracle, element by element, through the C ABI.
+Tolerances (bf16 inputs, fp32 accumulation): O max-abs <= 2e-2, mean-abs <= 2e-3, lse max-abs <= 5e-3."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import focus_oracle as fo
+from paper_2604_03260_b200 import binding as fb
+from paper_2604_03260_b200 import inputs as fi
+from tests.gpu_util import as_u32, assert_parity, compare_rows, gpu_assign, gpu_attn, gpu_tiles
+from tests.test_gpu_tiles import random_masks
+
+pytestmark = pytest.mark.gpu
+
+
+def oracle_masks(wl, Q, K, C):
+    mq, _ = fo.assign(fi.bf16_bits(Q), C.cpu().numpy(), wl.topk)
+    mk, _ = fo.assign(fi.bf16_bits(K), C.cpu().numpy(), wl.topk)
+    return mq, mk
+
+
+def to_dev(m):
+    return torch.from_numpy(m.view(np.int32)).cuda()
+
+
+def run_case(wl, layout=0, masks=None, rows=None, dense=False, impl=None):
+    Q, K, V, C = fi.make_inputs(wl, "cuda")
+    if masks is None:
+        mq, mk = oracle_masks(wl, Q, K, C)
+    else:
+        mq, mk = masks
+    old = os.environ.pop("FOCUS_ATTN_IMPL", None)
+    if impl:
+        os.environ["FOCUS_ATTN_IMPL"] = impl
+    try:
+        if dense:
+            O, lse = gpu_attn(wl, Q, K, V)
+        else:
+            dq, dk = to_dev(mq), to_dev(mk)
+            ws, _ = gpu_tiles(wl, dq, dk, layout)
+            O, lse = gpu_attn(wl, Q, K, V, dq, dk, ws, layout)
+    finally:
+        os.environ.pop("FOCUS_ATTN_IMPL", None)
+        if old is not None:
+            os.environ["FOCUS_ATTN_IMPL"] = old
+    stats = compare_rows(wl, Q, K, V, mq, mk, O, lse, rows=rows, dense=dense)
+    assert_parity(stats)
+    return stats
+
+
+@pytest.mark.parametrize("D", [64, 128, 256])
+def test_debug_kernel_matches_oracle(D):
+    wl = fi.Workload("s", 4, 2, D, 333, 4, 2, 17, seed=D)
+    run_case(wl, impl="simple")
+    run_case(wl, impl="simple", dense=True)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("n", [1, 100, 128, 129, 256, 257, 640, 1111])
+def test_dense_causal_mode(D, n):
+    wl = fi.Workload("d", 4, 2, D, n, 4, 2, 0, seed=n + D)
+    run_case(wl, dense=True)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("n,w,K,t", [(1, 0, 4, 2), (130, 0, 4, 1), (300, 7, 4, 2), (777, 128, 8, 2), (1000, 64, 4, 2),
+                                     (1500, 127, 4, 1), (1500, 129, 2, 1), (2048, 256, 4, 2), (2500, 5000, 4, 1),
+                                     (1300, 300, 32, 3), (1024, 64, 1, 1)])
+def test_original_layout_random_masks(D, n, w, K, t):
+    wl = fi.Workload("o", 4, 2, D, n, K, t, w, seed=n + w + D)
+    run_case(wl)
+
+
+@pytest.mark.parametrize("w,K", [(0, 4), (100, 4), (300, 8)])
+def test_original_layout_skips_dead_tiles(w, K):
+    """run-structured masks: whole far tiles die (skipped), others are full (mask-free)"""
+    wl = fi.Workload("b", 4, 2, 128, 4000, K, 1, w, seed=w + K)
+    rng = np.random.default_rng(w)
+    masks = (random_masks(rng, 4, wl.n, K, 1, True), random_masks(rng, 2, wl.n, K, 1, True))
+    run_case(wl, masks=masks)
+
+
+def test_softcap():
+    wl = fi.Workload("c", 4, 2, 128, 900, 4, 2, 50, softcap=5.0, scale=0.25, seed=3)
+    run_case(wl)
+    run_case(wl, dense=True)
+
+
+def test_strided_tensors_and_determinism():
+    wl = fi.Workload("st", 4, 2, 128, 700, 4, 2, 33, seed=12)
+    Q, K, V, C = fi.make_inputs(wl, "cuda")
+    mq, mk = oracle_masks(wl, Q, K, C)
+    dq, dk = to_dev(mq), to_dev(mk)
+    ws, _ = gpu_tiles(wl, dq, dk, 0)
+    O1, l1 = gpu_attn(wl, Q, K, V, dq, dk, ws, 0)
+    O2, l2 = gpu_attn(wl, Q, K, V, dq, dk, ws, 0)
+    assert torch.equal(O1, O2) and torch.equal(l1, l2)
+    tr = lambda x: x.transpose(0, 1).contiguous().transpose(0, 1)       # [n, H, D] storage
+    O3, l3 = gpu_attn(wl, tr(Q), tr(K), tr(V), dq, dk, ws, 0)
+    assert torch.equal(O1, O3) and torch.equal(l1, l3)
+
+
+def test_cfg1_all_rows_end_to_end():
+    """assign -> build_tiles -> attn on the GPU; the oracle attends with the GPU's masks, and the
+    masks themselves are compared (near-ties excepted) in test_gpu_assign"""
+    wl = fi.WORKLOADS["cfg1"]
+    Q, K, V, C = fi.make_inputs(wl, "cuda")
+    mq, _ = gpu_assign(wl, Q, C, wl.Hq)
+    mk, _ = gpu_assign(wl, K, C, wl.Hkv)
+    ws, _ = gpu_tiles(wl, mq, mk, 0)
+    O, lse = gpu_attn(wl, Q, K, V, mq, mk, ws, 0)
+    assert_parity(compare_rows(wl, Q, K, V, as_u32(mq), as_u32(mk), O, lse))
+    Od, lsed = gpu_attn(wl, Q, K, V)
+    assert_parity(compare_rows(wl, Q, K, V, as_u32(mq), as_u32(mk), Od, lsed, dense=True))
+
+
+def test_cfg2_two_heads_all_rows_others_sampled():
+    wl = fi.WORKLOADS["cfg2"]
+    Q, K, V, C = fi.make_inputs(wl, "cuda")
+    mq, mk = oracle_masks(wl, Q, K, C)
+    dq, dk = to_dev(mq), to_dev(mk)
+    ws, _ = gpu_tiles(wl, dq, dk, 0)
+    O, lse = gpu_attn(wl, Q, K, V, dq, dk, ws, 0)
+    rows = [np.stack([np.full(wl.n, h), np.arange(wl.n)], 1) for h in (0, 31)]
+    rows.append(fi.sample_rows(wl, 48))
+    assert_parity(compare_rows(wl, Q, K, V, mq, mk, O, lse, rows=np.concatenate(rows)))
