@@ -180,6 +180,29 @@ FOCUS_API int focus_count_kept(const focus_shape* shape, const uint32_t* mq, con
                      unsigned long long* counts_out, void* stream);
 
 /*
+ * focus_count_kept_noalloc -- the paper has no counterpart; this is a convenience of the library.
+ * Same result as focus_count_kept, for callers that cannot allocate device memory: code that was
+ * handed its input and output buffers by a host framework and owns no allocator, a server whose
+ * device arena is fully committed at start-up, or a latency-critical loop in which cudaMalloc is
+ * off limits because it synchronises the device.  Instead of reading the group bitmaps from a
+ * caller-allocated tiles workspace, this entry point builds them from mk into a fixed array that is
+ * part of the library image (FOCUS_NOALLOC_MAX_BYTES, resident on every device that loads the
+ * library until the process exits).  It calls no allocating routine.
+ *   mq          device, uint32 [batch*Hq, n]       mk   device, uint32 [batch*Hkv, n]
+ *   counts_out  device uint64 [batch*Hq]; overwritten
+ * Limit: batch*Hkv*ceil(n/128)*K*16 bytes must fit in FOCUS_NOALLOC_MAX_BYTES, otherwise
+ * FOCUS_ERR_CAPACITY is returned and nothing is launched (1 MiB covers the 128K-token metric point:
+ * 8 KV heads x 1024 tiles x 4 groups x 16 B = 512 KiB).
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call outside any stream capture.  All calls share the one array, which keeps the
+ * previous call's contents; each call rewrites the part it reads, so stale contents are harmless,
+ * but two calls whose kernels may overlap on the GPU (different streams) race on it.
+ */
+#define FOCUS_NOALLOC_MAX_BYTES (1 << 20)
+FOCUS_API int focus_count_kept_noalloc(const focus_shape* shape, const uint32_t* mq, const uint32_t* mk,
+                                       unsigned long long* counts_out, void* stream);
+
+/*
  * focus_selftest_umma -- diagnostic, not on the hot path (the paper has no counterpart): one
  * 128 x 128 x D tile S = A B^T and one 128 x D x 128 tile O = P V through the same TMA, descriptor
  * and tcgen05 building blocks as focus_attn_fwd, so that an encoding mistake shows up in isolation.

@@ -73,6 +73,8 @@ def lib():
                                      vp, vp]
         L.focus_count_kept.restype = C.c_int
         L.focus_count_kept.argtypes = [SP, vp, vp, vp, vp]
+        L.focus_count_kept_noalloc.restype = C.c_int
+        L.focus_count_kept_noalloc.argtypes = [SP, vp, vp, vp, vp]
         L.focus_selftest_umma.restype = C.c_int
         L.focus_selftest_umma.argtypes = [i32, vp, vp, vp, vp, vp, vp, vp, vp]
         _lib = L
@@ -143,6 +145,12 @@ def focus_attn_fwd(shape, q, k, v, mq, mk, tiles_ws, layout, o, lse, dev_status=
 
 def focus_count_kept(shape, mq, tiles_ws, counts_out, stream=None):
     _check(lib().focus_count_kept(C.byref(shape), _p(mq), _p(tiles_ws), _p(counts_out), _stream(stream)))
+
+
+def focus_count_kept_noalloc(shape, mq, mk, counts_out, stream=None):
+    """focus_count_kept for callers that may not allocate: the group bitmaps go to an array built into the
+    library (at most 1 MiB: batch*Hkv*ceil(n/128)*K*16 bytes), no workspace argument."""
+    _check(lib().focus_count_kept_noalloc(C.byref(shape), _p(mq), _p(mk), _p(counts_out), _stream(stream)))
 
 
 def focus_selftest_umma(D, a, b, p, v, s_out, o_out, dev_status, stream=None):
