@@ -12,6 +12,10 @@
 // the other run.  The running maximum is raised lazily (only when it grows by more than 2^8), and
 // then the owner of the row rescales its O row in TMEM itself.
 //
+// Head dimension 256 does not leave room in TMEM for two query tiles (O alone is 256 columns), so
+// there an item is a single 128-row query tile, S is double-buffered over consecutive key tiles
+// and one warpgroup does the softmax while the MMAs of the neighbouring tiles run.
+//
 // Which key tiles are visited: in dense mode every tile up to the diagonal; with a tiles
 // workspace, far tiles (every pair beyond the window) only when the live bitmap says the OR of the
 // query-tile masks meets the OR of the key-tile masks; near tiles always.
@@ -23,14 +27,13 @@ namespace focus {
 
 using namespace ptx;
 
-constexpr int ATT_THREADS = 384;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 constexpr float RESCALE_THRESHOLD = 8.0f;   // log2 units: the stale maximum may lag by a factor of 256
 
 struct AttnParams {
     int B, Hq, Hkv, G, n, w, K;
-    int nqb;                 // 256-row query blocks per head
+    int nqb;                 // items per head: 256-row query blocks (128-row tiles when D = 256)
     int nqt, nkt, nkw;
     int dense;
     float scale, softcap;
@@ -55,9 +58,9 @@ struct TileWalk {
     uint32_t bits;
     bool far_phase;
 
-    __device__ __forceinline__ void init(const AttnParams& p, int hq, int A) {
-        const int a0 = 2 * A;
-        const long long last_row = min((long long)p.n, (long long)(A + 1) * 256) - 1;
+    // a0 = first 128-row query tile of the item, nq = number of query tiles of the item (1 or 2)
+    __device__ __forceinline__ void init(const AttnParams& p, int hq, int a0, int nq) {
+        const long long last_row = min((long long)p.n, (long long)(a0 + nq) * 128) - 1;
         b_last = (int)(last_row / 128);
         f0 = 0;
         l0 = l1 = nullptr;
@@ -65,7 +68,7 @@ struct TileWalk {
             const long long d = (long long)a0 * 128 - p.w;
             f0 = d > 0 ? (int)(d / 128) : 0;
             l0 = p.live + ((size_t)hq * p.nqt + a0) * p.nkw;
-            if (a0 + 1 < p.nqt) l1 = l0 + p.nkw;
+            if (nq > 1 && a0 + 1 < p.nqt) l1 = l0 + p.nkw;
         }
         far_phase = f0 > 0;
         wd = -1;
@@ -96,17 +99,20 @@ struct TileWalk {
 
 template <int D>
 struct AttnCfg {
+    static constexpr int NQ = (D == 256) ? 1 : 2;            // 128-row query tiles per item
     static constexpr int SUBT = D / 64;
     static constexpr uint32_t SUB_BYTES = 128 * 64 * 2;
     static constexpr uint32_t TILE_BYTES = SUB_BYTES * SUBT;
-    static constexpr int NSTAGE = (D == 128) ? 5 : 8;
-    static constexpr uint32_t SMEM_BYTES = 1024 + 2 * TILE_BYTES + NSTAGE * TILE_BYTES;
+    static constexpr int NSTAGE = (D == 256) ? 2 : ((D == 128) ? 5 : 8);
+    static constexpr uint32_t SMEM_BYTES = 1024 + NQ * TILE_BYTES + NSTAGE * TILE_BYTES;
     static constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O0 = 256, COL_O1 = 256 + D;
+    static constexpr int THREADS = 128 + 128 * NQ;
 };
 
 struct SharedCtl {
     uint64_t q_full, q_empty;
     uint64_t s_full[2], p_full[2], o_full[2];
+    uint64_t pv_done;
     uint64_t kv_full[8], kv_empty[8];
     uint32_t tmem_base;
     int abort_flag;
@@ -135,22 +141,78 @@ __device__ __forceinline__ void report_timeout(const AttnParams& p, SharedCtl* c
     }
 }
 
+// Per-row 128-bit keep bitmap of one (query tile, key tile) pair.  Returns false when the tile needs
+// no mask at all; `all_masked` is set when no pair of the tile can be attended.
+struct TileMask {
+    uint32_t kw[4];
+    bool masked, all_masked;
+};
+
+__device__ __forceinline__ void build_tile_mask(TileMask& tm, const AttnParams& p, int a, int kb, long long i,
+                                                uint32_t mi, uint32_t aq, int f_x, int hk) {
+    const long long c0 = (long long)kb * 128;
+    const long long r_first = (long long)a * 128, r_last = r_first + 127;
+    tm.all_masked = c0 > r_last || r_first >= p.n;
+    const bool need_causal = c0 + 127 > r_first;
+    bool need_group = false, need_window = false;
+    if (!p.dense && !tm.all_masked) {
+        if (kb < f_x) {
+            need_group = !(aq & __ldg(p.andk + (size_t)hk * p.nkt + kb));
+        } else if (r_last - c0 > p.w) {
+            need_group = need_window = true;
+        }
+    }
+    tm.masked = need_causal || need_group;
+    tm.kw[0] = tm.kw[1] = tm.kw[2] = tm.kw[3] = 0xffffffffu;
+    if (tm.masked && !tm.all_masked) {
+        uint32_t sh[4] = {0, 0, 0, 0};
+        if (need_group) {
+            const uint32_t* gb = p.gbits + ((size_t)hk * p.nkt + kb) * p.K * 4;
+            for (uint32_t rem = mi; rem; rem &= rem - 1) {
+                const int g = __ffs(rem) - 1;
+                if (g < p.K) {
+                    const uint4 t = __ldg(reinterpret_cast<const uint4*>(gb + g * 4));
+                    sh[0] |= t.x; sh[1] |= t.y; sh[2] |= t.z; sh[3] |= t.w;
+                }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            uint32_t keep = 0xffffffffu;
+            if (need_group) {
+                keep = sh[q];
+                if (need_window) {
+                    const long long lo = i - p.w - c0 - 32 * q;          // columns >= lo are inside the window
+                    keep |= lo <= 0 ? 0xffffffffu : (lo >= 32 ? 0u : ~((1u << (int)lo) - 1u));
+                }
+            }
+            if (need_causal) {
+                const long long nk = i - c0 + 1 - 32 * q;                // columns < nk are causal
+                keep &= nk >= 32 ? 0xffffffffu : (nk <= 0 ? 0u : ((1u << (int)nk) - 1u));
+            }
+            tm.kw[q] = keep;
+        }
+    }
+}
+
 template <int D, bool SOFTCAP>
-__global__ void __launch_bounds__(ATT_THREADS, 1)
+__global__ void __launch_bounds__(AttnCfg<D>::THREADS, 1)
 focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
     using C = AttnCfg<D>;
+    constexpr int NQ = C::NQ;
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) SharedCtl ctl;
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sq = base;                                // 2 query tiles
-    const uint32_t skv = base + 2 * C::TILE_BYTES;            // ring of K / V tiles
+    const uint32_t sq = base;                                 // NQ query tiles
+    const uint32_t skv = base + NQ * C::TILE_BYTES;            // ring of K / V tiles
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int HQ = p.B * p.Hq;
 
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&ctl.q_full), 1);
         mbar_init(smem_u32(&ctl.q_empty), 1);
+        mbar_init(smem_u32(&ctl.pv_done), 1);
         for (int x = 0; x < 2; ++x) {
             mbar_init(smem_u32(&ctl.s_full[x]), 1);
             mbar_init(smem_u32(&ctl.p_full[x]), 128);
@@ -184,13 +246,13 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 const int hq = (int)(item % HQ);
                 const int b = hq / p.Hq, h = hq % p.Hq, hk = h / p.G;
                 if (it > 0 && !ctl_wait(&ctl.q_empty, (it - 1) & 1, &ctl)) { report_timeout(p, &ctl, 10, (int)item); break; }
-                mbar_arrive_expect_tx(smem_u32(&ctl.q_full), 2 * C::TILE_BYTES);
-                for (int x = 0; x < 2; ++x)
+                mbar_arrive_expect_tx(smem_u32(&ctl.q_full), NQ * C::TILE_BYTES);
+                for (int x = 0; x < NQ; ++x)
                     for (int c = 0; c < C::SUBT; ++c)
                         tma_load_4d(sq + x * C::TILE_BYTES + c * C::SUB_BYTES, &tm_q, smem_u32(&ctl.q_full), c * 64,
-                                    A * 256 + x * 128, h, b);
+                                    (A * NQ + x) * 128, h, b);
                 TileWalk walk;
-                walk.init(p, hq, A);
+                walk.init(p, hq, A * NQ, NQ);
                 int kb;
                 while (ok && (kb = walk.next()) >= 0) {
                     for (int kv = 0; kv < 2; ++kv) {
@@ -218,11 +280,13 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             constexpr uint32_t IDESC_S = idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t IDESC_O = idesc_bf16(128, D, 0, 1);
             long long nuse = 0;             // K/V stages consumed so far
-            uint32_t np[2] = {0, 0};        // P tiles consumed per query tile
+            uint32_t np[2] = {0, 0};        // P tiles consumed per S/P buffer
+            uint32_t gs = 0, gp = 0;        // NQ == 1: S tiles issued / P tiles consumed (buffer = count & 1)
             int it = 0;
             bool ok = true;
-            auto issue_s = [&](int x, uint32_t kaddr) {
-                const uint32_t d = tmem + (x ? C::COL_S1 : C::COL_S0);
+            // S[buf] = Q_x K^T
+            auto issue_s = [&](int x, int buf, uint32_t kaddr) {
+                const uint32_t d = tmem + (buf ? C::COL_S1 : C::COL_S0);
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t off = (ks / 4) * C::SUB_BYTES + (ks % 4) * 32;
@@ -230,73 +294,94 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             smem_desc_sw128(kaddr + off, 16, 1024), IDESC_S, ks > 0);
                 }
             };
-            auto issue_o = [&](int x, uint32_t vaddr, bool first) {
+            // O_x (+)= P[buf] V
+            auto issue_o = [&](int x, int buf, uint32_t vaddr, bool first) {
                 const uint32_t d = tmem + (x ? C::COL_O1 : C::COL_O0);
-                const uint32_t a = tmem + (x ? C::COL_S1 : C::COL_S0);
+                const uint32_t a = tmem + (buf ? C::COL_S1 : C::COL_S0);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
                     umma_ts(d, a + ks * 8, smem_desc_sw128(vaddr + ks * 2048, C::SUB_BYTES, 1024), IDESC_O,
                             (!first) || ks > 0);
             };
+            auto wait_kv = [&](int& slot, int where, int item) -> bool {
+                slot = (int)(nuse % C::NSTAGE);
+                if (!ctl_wait(&ctl.kv_full[slot], (uint32_t)((nuse / C::NSTAGE) & 1), &ctl)) {
+                    report_timeout(p, &ctl, where, item);
+                    return false;
+                }
+                ++nuse;
+                return true;
+            };
             for (long long item = blockIdx.x; ok && item < p.nitems; item += gridDim.x, ++it) {
                 const int A = p.nqb - 1 - (int)(item / HQ);
                 const int hq = (int)(item % HQ);
                 TileWalk walk;
-                walk.init(p, hq, A);
+                walk.init(p, hq, A * NQ, NQ);
                 int cur = walk.next();
                 if (!ctl_wait(&ctl.q_full, it & 1, &ctl)) { report_timeout(p, &ctl, 20, (int)item); break; }
-                // S of the first tile for both query tiles
-                {
-                    const int slot = (int)(nuse % C::NSTAGE);
-                    if (!ctl_wait(&ctl.kv_full[slot], (uint32_t)((nuse / C::NSTAGE) & 1), &ctl)) {
-                        report_timeout(p, &ctl, 21, (int)item); break;
-                    }
-                    tc_fence_after();
+                int slot;
+                if (!wait_kv(slot, 21, (int)item)) break;
+                tc_fence_after();
+                if constexpr (NQ == 2) {
                     const uint32_t kaddr = skv + slot * C::TILE_BYTES;
-                    issue_s(0, kaddr); umma_commit(smem_u32(&ctl.s_full[0]));
-                    issue_s(1, kaddr); umma_commit(smem_u32(&ctl.s_full[1]));
+                    issue_s(0, 0, kaddr); umma_commit(smem_u32(&ctl.s_full[0]));
+                    issue_s(1, 1, kaddr); umma_commit(smem_u32(&ctl.s_full[1]));
                     umma_commit(smem_u32(&ctl.kv_empty[slot]));
-                    ++nuse;
+                } else {
+                    issue_s(0, gs & 1, skv + slot * C::TILE_BYTES);
+                    umma_commit(smem_u32(&ctl.s_full[gs & 1]));
+                    umma_commit(smem_u32(&ctl.kv_empty[slot]));
+                    ++gs;
                 }
                 bool first = true;
                 while (cur >= 0) {
                     const int nxt = walk.next();
-                    const int vslot = (int)(nuse % C::NSTAGE);
-                    if (!ctl_wait(&ctl.kv_full[vslot], (uint32_t)((nuse / C::NSTAGE) & 1), &ctl)) {
-                        report_timeout(p, &ctl, 22, (int)item); ok = false; break;
-                    }
-                    ++nuse;
+                    int vslot, kslot = 0;
+                    if (!wait_kv(vslot, 22, (int)item)) { ok = false; break; }
                     const uint32_t vaddr = skv + vslot * C::TILE_BYTES;
-                    int kslot = 0;
                     uint32_t kaddr = 0;
                     if (nxt >= 0) {
-                        kslot = (int)(nuse % C::NSTAGE);
-                        if (!ctl_wait(&ctl.kv_full[kslot], (uint32_t)((nuse / C::NSTAGE) & 1), &ctl)) {
-                            report_timeout(p, &ctl, 23, (int)item); ok = false; break;
-                        }
-                        ++nuse;
+                        if (!wait_kv(kslot, 23, (int)item)) { ok = false; break; }
                         kaddr = skv + kslot * C::TILE_BYTES;
                     } else {
                         umma_commit(smem_u32(&ctl.q_empty));     // every S of this item has been issued
                     }
-                    // query tile 0
-                    if (!ctl_wait(&ctl.p_full[0], np[0] & 1, &ctl)) { report_timeout(p, &ctl, 24, (int)item); ok = false; break; }
-                    ++np[0];
-                    tc_fence_after();
-                    issue_o(0, vaddr, first);
-                    if (nxt >= 0) { issue_s(0, kaddr); umma_commit(smem_u32(&ctl.s_full[0])); }
-                    else umma_commit(smem_u32(&ctl.o_full[0]));
-                    // query tile 1
-                    if (!ctl_wait(&ctl.p_full[1], np[1] & 1, &ctl)) { report_timeout(p, &ctl, 25, (int)item); ok = false; break; }
-                    ++np[1];
-                    tc_fence_after();
-                    issue_o(1, vaddr, first);
-                    umma_commit(smem_u32(&ctl.kv_empty[vslot]));
-                    if (nxt >= 0) {
-                        issue_s(1, kaddr); umma_commit(smem_u32(&ctl.s_full[1]));
-                        umma_commit(smem_u32(&ctl.kv_empty[kslot]));
+                    if constexpr (NQ == 2) {
+                        // query tile 0
+                        if (!ctl_wait(&ctl.p_full[0], np[0] & 1, &ctl)) { report_timeout(p, &ctl, 24, (int)item); ok = false; break; }
+                        ++np[0];
+                        tc_fence_after();
+                        issue_o(0, 0, vaddr, first);
+                        if (nxt >= 0) { issue_s(0, 0, kaddr); umma_commit(smem_u32(&ctl.s_full[0])); }
+                        else umma_commit(smem_u32(&ctl.o_full[0]));
+                        // query tile 1
+                        if (!ctl_wait(&ctl.p_full[1], np[1] & 1, &ctl)) { report_timeout(p, &ctl, 25, (int)item); ok = false; break; }
+                        ++np[1];
+                        tc_fence_after();
+                        issue_o(1, 1, vaddr, first);
+                        umma_commit(smem_u32(&ctl.kv_empty[vslot]));
+                        if (nxt >= 0) {
+                            issue_s(1, 1, kaddr); umma_commit(smem_u32(&ctl.s_full[1]));
+                            umma_commit(smem_u32(&ctl.kv_empty[kslot]));
+                        } else {
+                            umma_commit(smem_u32(&ctl.o_full[1]));
+                        }
                     } else {
-                        umma_commit(smem_u32(&ctl.o_full[1]));
+                        // S of the next tile goes to the other buffer before this tile's PV is issued
+                        if (nxt >= 0) {
+                            issue_s(0, gs & 1, kaddr);
+                            umma_commit(smem_u32(&ctl.s_full[gs & 1]));
+                            umma_commit(smem_u32(&ctl.kv_empty[kslot]));
+                            ++gs;
+                        }
+                        const int buf = gp & 1;
+                        if (!ctl_wait(&ctl.p_full[buf], (gp >> 1) & 1, &ctl)) { report_timeout(p, &ctl, 26, (int)item); ok = false; break; }
+                        ++gp;
+                        tc_fence_after();
+                        issue_o(0, buf, vaddr, first);
+                        umma_commit(smem_u32(&ctl.kv_empty[vslot]));
+                        umma_commit(smem_u32(&ctl.pv_done));
+                        if (nxt < 0) umma_commit(smem_u32(&ctl.o_full[0]));
                     }
                     first = false;
                     cur = nxt;
@@ -306,14 +391,13 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         __syncwarp();
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ softmax + epilogue
-        const int x = (warp - 4) >> 2;                       // query tile of this warpgroup
+        const int x = (warp - 4) >> 2;                       // query tile of this warpgroup (0 when NQ == 1)
         const int row_in_tile = ((warp & 3) << 5) | lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t t_s = tmem + lane_base + (x ? C::COL_S1 : C::COL_S0);
         const uint32_t t_o = tmem + lane_base + (x ? C::COL_O1 : C::COL_O0);
         const float sl2 = SOFTCAP ? LOG2E : p.scale * LOG2E;
         const float cap_in = SOFTCAP ? p.scale / p.softcap : 0.f;
-        uint32_t ns = 0;
+        uint32_t ns = 0;                                     // S tiles consumed by this warpgroup
         int it = 0;
         bool ok = true;
         for (long long item = blockIdx.x; ok && item < p.nitems; item += gridDim.x, ++it) {
@@ -321,71 +405,29 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             const int hq = (int)(item % HQ);
             const int bb = hq / p.Hq, h = hq % p.Hq;
             const int hk = bb * p.Hkv + h / p.G;
-            const int a = 2 * A + x;
+            const int a = A * NQ + x;
             const long long i = (long long)a * 128 + row_in_tile;
             const bool valid = i < p.n;
             const uint32_t mi = (valid && !p.dense) ? __ldg(p.mq + (size_t)hq * p.n + i) : 0u;
             const uint32_t aq = (!p.dense && a < p.nqt) ? __ldg(p.andq + (size_t)hq * p.nqt + a) : 0u;
             const long long dfar = (long long)a * 128 - p.w;
             const int f_x = (!p.dense && dfar > 0) ? (int)(dfar / 128) : 0;   // tiles b < f_x are far for this query tile
-            const long long r_last = (long long)a * 128 + 127;
             float m_used = -INFINITY, l = 0.f;
             TileWalk walk;
-            walk.init(p, hq, A);
+            walk.init(p, hq, A * NQ, NQ);
             int kb;
             bool first = true;
             while ((kb = walk.next()) >= 0) {
-                const long long c0 = (long long)kb * 128;
-                // ---- how this tile is masked for this query tile (uniform over the warpgroup)
-                bool all_masked = c0 > r_last || (long long)a * 128 >= p.n;
-                bool need_causal = c0 + 127 > (long long)a * 128;
-                bool need_group = false, need_window = false;
-                if (!p.dense && !all_masked) {
-                    if (kb < f_x) {
-                        need_group = !(aq & __ldg(p.andk + (size_t)hk * p.nkt + kb));
-                    } else if (r_last - c0 > p.w) {
-                        need_group = need_window = true;
-                    }
-                }
-                uint32_t kw[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
-                const bool masked = need_causal || need_group;
-                if (masked && !all_masked) {
-                    uint32_t sh[4] = {0, 0, 0, 0};
-                    if (need_group) {
-                        const uint32_t* gb = p.gbits + ((size_t)hk * p.nkt + kb) * p.K * 4;
-                        uint32_t rem = mi;
-                        while (rem) {
-                            const int g = __ffs(rem) - 1;
-                            rem &= rem - 1;
-                            if (g < p.K) {
-                                const uint4 t = __ldg(reinterpret_cast<const uint4*>(gb + g * 4));
-                                sh[0] |= t.x; sh[1] |= t.y; sh[2] |= t.z; sh[3] |= t.w;
-                            }
-                        }
-                    }
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        uint32_t keep = 0xffffffffu;
-                        if (need_group) {
-                            keep = sh[q];
-                            if (need_window) {
-                                const long long lo = i - p.w - c0 - 32 * q;      // columns >= lo are inside the window
-                                keep |= lo <= 0 ? 0xffffffffu : (lo >= 32 ? 0u : ~((1u << (int)lo) - 1u));
-                            }
-                        }
-                        if (need_causal) {
-                            const long long nk = i - c0 + 1 - 32 * q;            // columns < nk are causal
-                            keep &= nk >= 32 ? 0xffffffffu : (nk <= 0 ? 0u : ((1u << (int)nk) - 1u));
-                        }
-                        kw[q] = keep;
-                    }
-                }
+                TileMask tm;
+                build_tile_mask(tm, p, a, kb, i, mi, aq, f_x, hk);
                 // ---- wait for S
-                if (!ctl_wait(&ctl.s_full[x], ns & 1, &ctl)) { report_timeout(p, &ctl, 30 + x, (int)item); ok = false; break; }
-                ++ns;
+                const int buf = NQ == 2 ? x : (int)(ns & 1);
+                const uint32_t par = NQ == 2 ? (ns & 1) : ((ns >> 1) & 1);
+                if (!ctl_wait(&ctl.s_full[buf], par, &ctl)) { report_timeout(p, &ctl, 30 + x, (int)item); ok = false; break; }
+                const uint32_t t_s = tmem + lane_base + (buf ? C::COL_S1 : C::COL_S0);
                 tc_fence_after();
                 uint32_t pk[64];
-                if (all_masked) {
+                if (tm.all_masked) {
 #pragma unroll
                     for (int c = 0; c < 64; ++c) pk[c] = 0u;
                 } else {
@@ -398,7 +440,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     for (int c = 0; c < 128; ++c) {
                         float s = __uint_as_float(sr[c]);
                         if (SOFTCAP) s = p.softcap * tanh_approx(s * cap_in);
-                        if (masked) s = ((kw[c >> 5] >> (c & 31)) & 1u) ? s : -INFINITY;
+                        if (tm.masked) s = ((tm.kw[c >> 5] >> (c & 31)) & 1u) ? s : -INFINITY;
                         sr[c] = __float_as_uint(s);
                         mt = fmaxf(mt, s);
                     }
@@ -414,7 +456,12 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         raise = true;
                     }
                     if (__any_sync(0xffffffffu, raise) && !first) {
-                        // the previous PV of this query tile has completed (its commit precedes s_full)
+                        // O may only be touched once the previous PV of this query tile has completed.  With two
+                        // query tiles its commit precedes s_full; with double-buffered S it has its own barrier.
+                        bool pv_ok = true;
+                        if constexpr (NQ == 1) pv_ok = ctl_wait(&ctl.pv_done, (ns - 1) & 1, &ctl);
+                        if (!pv_ok) { report_timeout(p, &ctl, 35, (int)item); ok = false; }
+                        tc_fence_after();
 #pragma unroll 1
                         for (int c = 0; c < D / 16; ++c) {
                             uint32_t ov[16];
@@ -442,8 +489,10 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 tmem_st32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(smem_u32(&ctl.p_full[x]));
+                mbar_arrive(smem_u32(&ctl.p_full[buf]));
+                ++ns;
                 first = false;
+                if (!ok) break;
             }
             if (!ok) break;
             // ---- epilogue: O / l -> bf16 -> global, lse
@@ -488,7 +537,7 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
     if ((rc = make_tmap_qkv(&tv, a.v, a.s.batch, a.s.Hkv, a.s.n, D))) return rc;
     AttnParams p;
     p.B = a.s.batch; p.Hq = a.s.Hq; p.Hkv = a.s.Hkv; p.G = a.s.Hq / a.s.Hkv; p.n = a.s.n; p.w = a.s.window; p.K = a.s.K;
-    p.nqb = cdiv(a.s.n, 256);
+    p.nqb = cdiv(a.s.n, 128 * C::NQ);
     p.nqt = cdiv(a.s.n, 128); p.nkt = cdiv(a.s.n, 128); p.nkw = cdiv(p.nkt, 32);
     p.dense = a.ws ? 0 : 1;
     p.scale = a.scale; p.softcap = a.s.softcap;
@@ -510,7 +559,7 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
                          "cudaFuncSetAttribute(attn)")))
         return rc;
     const int grid = (int)(p.nitems < sms ? p.nitems : sms);
-    kern<<<grid, ATT_THREADS, C::SMEM_BYTES, st>>>(tq, tk, tv, p);
+    kern<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, tk, tv, p);
     return check_cuda(cudaGetLastError(), "attention kernel launch");
 }
 
@@ -521,8 +570,9 @@ int launch_attn_sm100(const AttnArgs& a, cudaStream_t st) {
     switch (a.s.D) {
         case 64: return cap ? launch_attn_t<64, true>(a, st) : launch_attn_t<64, false>(a, st);
         case 128: return cap ? launch_attn_t<128, true>(a, st) : launch_attn_t<128, false>(a, st);
+        case 256: return cap ? launch_attn_t<256, true>(a, st) : launch_attn_t<256, false>(a, st);
     }
-    return fail(FOCUS_ERR_UNSUPPORTED, "head dimension %d is not available in the tensor-core kernel yet", a.s.D);
+    return fail(FOCUS_ERR_UNSUPPORTED, "D (%d) must be 64, 128 or 256", a.s.D);
 }
 
 }  // namespace focus

@@ -57,14 +57,14 @@ def test_debug_kernel_matches_oracle(D):
     run_case(wl, impl="simple", dense=True)
 
 
-@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("D", [64, 128, 256])
 @pytest.mark.parametrize("n", [1, 100, 128, 129, 256, 257, 640, 1111])
 def test_dense_causal_mode(D, n):
     wl = fi.Workload("d", 4, 2, D, n, 4, 2, 0, seed=n + D)
     run_case(wl, dense=True)
 
 
-@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("D", [64, 128, 256])
 @pytest.mark.parametrize("n,w,K,t", [(1, 0, 4, 2), (130, 0, 4, 1), (300, 7, 4, 2), (777, 128, 8, 2), (1000, 64, 4, 2),
                                      (1500, 127, 4, 1), (1500, 129, 2, 1), (2048, 256, 4, 2), (2500, 5000, 4, 1),
                                      (1300, 300, 32, 3), (1024, 64, 1, 1)])
@@ -73,19 +73,23 @@ def test_original_layout_random_masks(D, n, w, K, t):
     run_case(wl)
 
 
+@pytest.mark.parametrize("D", [128, 256])
 @pytest.mark.parametrize("w,K", [(0, 4), (100, 4), (300, 8)])
-def test_original_layout_skips_dead_tiles(w, K):
+def test_original_layout_skips_dead_tiles(w, K, D):
     """run-structured masks: whole far tiles die (skipped), others are full (mask-free)"""
-    wl = fi.Workload("b", 4, 2, 128, 4000, K, 1, w, seed=w + K)
+    wl = fi.Workload("b", 4, 2, D, 4000, K, 1, w, seed=w + K)
     rng = np.random.default_rng(w)
     masks = (random_masks(rng, 4, wl.n, K, 1, True), random_masks(rng, 2, wl.n, K, 1, True))
     run_case(wl, masks=masks)
 
 
-def test_softcap():
-    wl = fi.Workload("c", 4, 2, 128, 900, 4, 2, 50, softcap=5.0, scale=0.25, seed=3)
+@pytest.mark.parametrize("D", [64, 128, 256])
+def test_softcap(D):
+    wl = fi.Workload("c", 4, 2, D, 900, 4, 2, 50, softcap=5.0, scale=0.25, seed=3)
     run_case(wl)
     run_case(wl, dense=True)
+    wl = fi.Workload("c50", 4, 2, D, 1500, 4, 1, 300, softcap=50.0, scale=1.0 / 16, seed=4)
+    run_case(wl)
 
 
 def test_strided_tensors_and_determinism():
