@@ -30,6 +30,42 @@ using namespace ptx;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 constexpr float RESCALE_THRESHOLD = 8.0f;   // log2 units: the stale maximum may lag by a factor of 256
+// Of every 8 consecutive probabilities, this many take their exponential from a polynomial on the
+// FMA/ALU pipes instead of the special-function unit, which would otherwise be as busy as the tensor pipe.
+constexpr int EX2_POLY_PER_8 = 0;
+// Registers per thread after the warps have split into roles (setmaxnreg): the load/MMA warpgroup
+// gives most of its share to the softmax warpgroups.
+constexpr int REGS_CONTROL = 96;
+constexpr int REGS_SOFTMAX_2WG = 200;        // 128*96 + 256*200 = 63488 <= 65536
+constexpr int REGS_SOFTMAX_1WG = 232;        // 128*96 + 128*232
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
+// 2^x for a pair of arguments in [-inf, 8] without the special-function unit: split x = n + f with
+// n = round(x) (magic-number addition), evaluate a cubic for 2^f on [-0.5, 0.5] (relative error
+// 7.5e-5, far below the bf16 rounding of the probabilities) and add n to the exponent field.
+// Arguments below -126 (masked pairs arrive as -inf) give 2^-126, which vanishes in every sum.
+__device__ __forceinline__ float2 ex2_poly2(float2 x) {
+    constexpr float MAGIC = 12582912.f;      // 1.5 * 2^23
+    x.x = fmaxf(x.x, -126.f);
+    x.y = fmaxf(x.y, -126.f);
+    const float2 t = __fadd2_rn(x, make_float2(MAGIC, MAGIC));
+    const float2 n = __fadd2_rn(t, make_float2(-MAGIC, -MAGIC));
+    const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
+    float2 p = __ffma2_rn(make_float2(0.0551716648f, 0.0551716648f), f, make_float2(0.2426111251f, 0.2426111251f));
+    p = __ffma2_rn(p, f, make_float2(0.6932609677f, 0.6932609677f));
+    p = __ffma2_rn(p, f, make_float2(0.9999280572f, 0.9999280572f));
+    float2 r;
+    r.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
+    r.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
+    return r;
+}
 
 struct AttnParams {
     int B, Hq, Hkv, G, n, w, K;
@@ -195,6 +231,25 @@ __device__ __forceinline__ void build_tile_mask(TileMask& tm, const AttnParams& 
     }
 }
 
+// Item order.  Items are laid out KV head by KV head, heaviest query block first inside a head
+// group, so that the CTAs running at the same time stream the K/V of one KV head through L2.  CTA c
+// takes position c of every even round of gridDim.x items and position gridDim.x-1-c of every odd
+// round, which cancels the cost gradient inside a round.  Returns false past the last item.
+struct Item { int A, bb, h, hq; long long id; };
+__device__ __forceinline__ bool item_of(const AttnParams& p, int round, Item& t) {
+    const int g = (int)gridDim.x, c = (int)blockIdx.x;
+    t.id = (long long)round * g + ((round & 1) ? g - 1 - c : c);
+    if (t.id >= p.nitems) return false;
+    const int per_group = p.nqb * p.G;
+    const int grp = (int)(t.id / per_group);              // batch * Hkv + KV head
+    const int rem = (int)(t.id % per_group);
+    t.A = p.nqb - 1 - rem / p.G;
+    t.bb = grp / p.Hkv;
+    t.h = (grp % p.Hkv) * p.G + rem % p.G;
+    t.hq = t.bb * p.Hq + t.h;
+    return true;
+}
+
 template <int D, bool SOFTCAP>
 __global__ void __launch_bounds__(AttnCfg<D>::THREADS, 1)
 focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -207,7 +262,6 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t sq = base;                                 // NQ query tiles
     const uint32_t skv = base + NQ * C::TILE_BYTES;            // ring of K / V tiles
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int HQ = p.B * p.Hq;
 
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&ctl.q_full), 1);
@@ -234,6 +288,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     tc_fence_after();
     const uint32_t tmem = ctl.tmem_base;
 
+    if (warp < 4) reg_dec<REGS_CONTROL>();
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -241,10 +296,10 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             long long nload = 0;
             int it = 0;
             bool ok = true;
-            for (long long item = blockIdx.x; ok && item < p.nitems; item += gridDim.x, ++it) {
-                const int A = p.nqb - 1 - (int)(item / HQ);
-                const int hq = (int)(item % HQ);
-                const int b = hq / p.Hq, h = hq % p.Hq, hk = h / p.G;
+            Item t;
+            for (; ok && item_of(p, it, t); ++it) {
+                const int A = t.A, hq = t.hq, b = t.bb, h = t.h, hk = h / p.G;
+                const long long item = t.id;
                 if (it > 0 && !ctl_wait(&ctl.q_empty, (it - 1) & 1, &ctl)) { report_timeout(p, &ctl, 10, (int)item); break; }
                 mbar_arrive_expect_tx(smem_u32(&ctl.q_full), NQ * C::TILE_BYTES);
                 for (int x = 0; x < NQ; ++x)
@@ -276,7 +331,9 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // The whole warp runs the loop (so that addresses and descriptors stay warp-uniform); one elected
+        // lane issues the MMAs and commits.
+        {
             constexpr uint32_t IDESC_S = idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t IDESC_O = idesc_bf16(128, D, 0, 1);
             long long nuse = 0;             // K/V stages consumed so far
@@ -284,24 +341,35 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             uint32_t gs = 0, gp = 0;        // NQ == 1: S tiles issued / P tiles consumed (buffer = count & 1)
             int it = 0;
             bool ok = true;
+            const uint64_t qdesc0 = smem_desc_sw128(sq, 16, 1024);
+            const uint64_t kvdesc0 = smem_desc_sw128(skv, 16, 1024);             // K tiles: K-major
+            const uint64_t vdesc0 = smem_desc_sw128(skv, C::SUB_BYTES, 1024);     // V tiles: MN-major
             // S[buf] = Q_x K^T
-            auto issue_s = [&](int x, int buf, uint32_t kaddr) {
-                const uint32_t d = tmem + (buf ? C::COL_S1 : C::COL_S0);
+            auto issue_s = [&](int x, int buf, int kslot) {
+                if (elect_one()) {
+                    const uint32_t d = tmem + (buf ? C::COL_S1 : C::COL_S0);
+                    const uint64_t ad = qdesc0 + (uint64_t)((x * C::TILE_BYTES) >> 4);
+                    const uint64_t bd = kvdesc0 + (uint64_t)((kslot * C::TILE_BYTES) >> 4);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks / 4) * C::SUB_BYTES + (ks % 4) * 32;
-                    umma_ss(d, smem_desc_sw128(sq + x * C::TILE_BYTES + off, 16, 1024),
-                            smem_desc_sw128(kaddr + off, 16, 1024), IDESC_S, ks > 0);
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint64_t off = (uint64_t)(((ks / 4) * C::SUB_BYTES + (ks % 4) * 32) >> 4);
+                        umma_ss(d, ad + off, bd + off, IDESC_S, ks > 0);
+                    }
                 }
             };
             // O_x (+)= P[buf] V
-            auto issue_o = [&](int x, int buf, uint32_t vaddr, bool first) {
-                const uint32_t d = tmem + (x ? C::COL_O1 : C::COL_O0);
-                const uint32_t a = tmem + (buf ? C::COL_S1 : C::COL_S0);
+            auto issue_o = [&](int x, int buf, int vslot, bool first) {
+                if (elect_one()) {
+                    const uint32_t d = tmem + (x ? C::COL_O1 : C::COL_O0);
+                    const uint32_t a = tmem + (buf ? C::COL_S1 : C::COL_S0);
+                    const uint64_t bd = vdesc0 + (uint64_t)((vslot * C::TILE_BYTES) >> 4);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    umma_ts(d, a + ks * 8, smem_desc_sw128(vaddr + ks * 2048, C::SUB_BYTES, 1024), IDESC_O,
-                            (!first) || ks > 0);
+                    for (int ks = 0; ks < 8; ++ks)
+                        umma_ts(d, a + ks * 8, bd + (uint64_t)((ks * 2048) >> 4), IDESC_O, (!first) || ks > 0);
+                }
+            };
+            auto commit = [&](uint64_t* bar) {
+                if (elect_one()) umma_commit(smem_u32(bar));
             };
             auto wait_kv = [&](int& slot, int where, int item) -> bool {
                 slot = (int)(nuse % C::NSTAGE);
@@ -312,9 +380,10 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 ++nuse;
                 return true;
             };
-            for (long long item = blockIdx.x; ok && item < p.nitems; item += gridDim.x, ++it) {
-                const int A = p.nqb - 1 - (int)(item / HQ);
-                const int hq = (int)(item % HQ);
+            Item t;
+            for (; ok && item_of(p, it, t); ++it) {
+                const int A = t.A, hq = t.hq;
+                const long long item = t.id;
                 TileWalk walk;
                 walk.init(p, hq, A * NQ, NQ);
                 int cur = walk.next();
@@ -323,14 +392,13 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (!wait_kv(slot, 21, (int)item)) break;
                 tc_fence_after();
                 if constexpr (NQ == 2) {
-                    const uint32_t kaddr = skv + slot * C::TILE_BYTES;
-                    issue_s(0, 0, kaddr); umma_commit(smem_u32(&ctl.s_full[0]));
-                    issue_s(1, 1, kaddr); umma_commit(smem_u32(&ctl.s_full[1]));
-                    umma_commit(smem_u32(&ctl.kv_empty[slot]));
+                    issue_s(0, 0, slot); commit(&ctl.s_full[0]);
+                    issue_s(1, 1, slot); commit(&ctl.s_full[1]);
+                    commit(&ctl.kv_empty[slot]);
                 } else {
-                    issue_s(0, gs & 1, skv + slot * C::TILE_BYTES);
-                    umma_commit(smem_u32(&ctl.s_full[gs & 1]));
-                    umma_commit(smem_u32(&ctl.kv_empty[slot]));
+                    issue_s(0, gs & 1, slot);
+                    commit(&ctl.s_full[gs & 1]);
+                    commit(&ctl.kv_empty[slot]);
                     ++gs;
                 }
                 bool first = true;
@@ -338,50 +406,47 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     const int nxt = walk.next();
                     int vslot, kslot = 0;
                     if (!wait_kv(vslot, 22, (int)item)) { ok = false; break; }
-                    const uint32_t vaddr = skv + vslot * C::TILE_BYTES;
-                    uint32_t kaddr = 0;
                     if (nxt >= 0) {
                         if (!wait_kv(kslot, 23, (int)item)) { ok = false; break; }
-                        kaddr = skv + kslot * C::TILE_BYTES;
                     } else {
-                        umma_commit(smem_u32(&ctl.q_empty));     // every S of this item has been issued
+                        commit(&ctl.q_empty);     // every S of this item has been issued
                     }
                     if constexpr (NQ == 2) {
                         // query tile 0
                         if (!ctl_wait(&ctl.p_full[0], np[0] & 1, &ctl)) { report_timeout(p, &ctl, 24, (int)item); ok = false; break; }
                         ++np[0];
                         tc_fence_after();
-                        issue_o(0, 0, vaddr, first);
-                        if (nxt >= 0) { issue_s(0, 0, kaddr); umma_commit(smem_u32(&ctl.s_full[0])); }
-                        else umma_commit(smem_u32(&ctl.o_full[0]));
+                        issue_o(0, 0, vslot, first);
+                        if (nxt >= 0) { issue_s(0, 0, kslot); commit(&ctl.s_full[0]); }
+                        else commit(&ctl.o_full[0]);
                         // query tile 1
                         if (!ctl_wait(&ctl.p_full[1], np[1] & 1, &ctl)) { report_timeout(p, &ctl, 25, (int)item); ok = false; break; }
                         ++np[1];
                         tc_fence_after();
-                        issue_o(1, 1, vaddr, first);
-                        umma_commit(smem_u32(&ctl.kv_empty[vslot]));
+                        issue_o(1, 1, vslot, first);
+                        commit(&ctl.kv_empty[vslot]);
                         if (nxt >= 0) {
-                            issue_s(1, 1, kaddr); umma_commit(smem_u32(&ctl.s_full[1]));
-                            umma_commit(smem_u32(&ctl.kv_empty[kslot]));
+                            issue_s(1, 1, kslot); commit(&ctl.s_full[1]);
+                            commit(&ctl.kv_empty[kslot]);
                         } else {
-                            umma_commit(smem_u32(&ctl.o_full[1]));
+                            commit(&ctl.o_full[1]);
                         }
                     } else {
                         // S of the next tile goes to the other buffer before this tile's PV is issued
                         if (nxt >= 0) {
-                            issue_s(0, gs & 1, kaddr);
-                            umma_commit(smem_u32(&ctl.s_full[gs & 1]));
-                            umma_commit(smem_u32(&ctl.kv_empty[kslot]));
+                            issue_s(0, gs & 1, kslot);
+                            commit(&ctl.s_full[gs & 1]);
+                            commit(&ctl.kv_empty[kslot]);
                             ++gs;
                         }
                         const int buf = gp & 1;
                         if (!ctl_wait(&ctl.p_full[buf], (gp >> 1) & 1, &ctl)) { report_timeout(p, &ctl, 26, (int)item); ok = false; break; }
                         ++gp;
                         tc_fence_after();
-                        issue_o(0, buf, vaddr, first);
-                        umma_commit(smem_u32(&ctl.kv_empty[vslot]));
-                        umma_commit(smem_u32(&ctl.pv_done));
-                        if (nxt < 0) umma_commit(smem_u32(&ctl.o_full[0]));
+                        issue_o(0, buf, vslot, first);
+                        commit(&ctl.kv_empty[vslot]);
+                        commit(&ctl.pv_done);
+                        if (nxt < 0) commit(&ctl.o_full[0]);
                     }
                     first = false;
                     cur = nxt;
@@ -391,19 +456,21 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         __syncwarp();
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ softmax + epilogue
+        if constexpr (NQ == 2) reg_inc<REGS_SOFTMAX_2WG>(); else reg_inc<REGS_SOFTMAX_1WG>();
         const int x = (warp - 4) >> 2;                       // query tile of this warpgroup (0 when NQ == 1)
         const int row_in_tile = ((warp & 3) << 5) | lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t t_o = tmem + lane_base + (x ? C::COL_O1 : C::COL_O0);
-        const float sl2 = SOFTCAP ? LOG2E : p.scale * LOG2E;
+        // logits in log2 units: sl2 * S, or with a softcap sl2 * tanh(cap_in * S)
+        const float sl2 = SOFTCAP ? p.softcap * LOG2E : p.scale * LOG2E;
         const float cap_in = SOFTCAP ? p.scale / p.softcap : 0.f;
         uint32_t ns = 0;                                     // S tiles consumed by this warpgroup
         int it = 0;
         bool ok = true;
-        for (long long item = blockIdx.x; ok && item < p.nitems; item += gridDim.x, ++it) {
-            const int A = p.nqb - 1 - (int)(item / HQ);
-            const int hq = (int)(item % HQ);
-            const int bb = hq / p.Hq, h = hq % p.Hq;
+        Item t;
+        for (; ok && item_of(p, it, t); ++it) {
+            const int A = t.A, hq = t.hq, bb = t.bb, h = t.h;
+            const long long item = t.id;
             const int hk = bb * p.Hkv + h / p.G;
             const int a = A * NQ + x;
             const long long i = (long long)a * 128 + row_in_tile;
@@ -435,16 +502,25 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
                     for (int c = 0; c < 4; ++c) tmem_ld32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[c * 32]));
                     tmem_wait_ld();
-                    float mt = -INFINITY;
+                    if (SOFTCAP) {
 #pragma unroll
-                    for (int c = 0; c < 128; ++c) {
-                        float s = __uint_as_float(sr[c]);
-                        if (SOFTCAP) s = p.softcap * tanh_approx(s * cap_in);
-                        if (tm.masked) s = ((tm.kw[c >> 5] >> (c & 31)) & 1u) ? s : -INFINITY;
-                        sr[c] = __float_as_uint(s);
-                        mt = fmaxf(mt, s);
+                        for (int c = 0; c < 128; ++c) sr[c] = __float_as_uint(tanh_approx(__uint_as_float(sr[c]) * cap_in));
                     }
-                    mt *= sl2;                                      // log2 units (sl2 > 0; -inf stays -inf)
+                    if (tm.masked) {
+#pragma unroll
+                        for (int c = 0; c < 128; ++c)
+                            sr[c] = ((tm.kw[c >> 5] >> (c & 31)) & 1u) ? sr[c] : 0xff800000u;      // -inf
+                    }
+                    // ---- row maximum of the tile: four independent chains of three-input maxima
+                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                    for (int c = 0; c < 128; c += 8) {
+                        mx0 = max3(mx0, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
+                        mx1 = max3(mx1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
+                        mx2 = max3(mx2, __uint_as_float(sr[c + 4]), __uint_as_float(sr[c + 5]));
+                        mx3 = max3(mx3, __uint_as_float(sr[c + 6]), __uint_as_float(sr[c + 7]));
+                    }
+                    const float mt = max3(mx0, mx1, fmaxf(mx2, mx3)) * sl2;   // log2 units (sl2 > 0; -inf stays -inf)
                     // ---- lazy maximum: raise the reference only when it lags by more than the threshold
                     float factor = 1.f;
                     bool raise = false;
@@ -474,16 +550,29 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     }
                     l *= factor;
                     const float msub = m_used == -INFINITY ? 0.f : m_used;
-                    float rs0 = 0.f, rs1 = 0.f;
+                    // ---- probabilities: packed fp32 pairs; part of the exponentials on the FMA/ALU pipes
+                    const float2 sl2v = make_float2(sl2, sl2), nmv = make_float2(-msub, -msub);
+                    float2 acc[4];
 #pragma unroll
-                    for (int c = 0; c < 128; c += 2) {
-                        const float p0 = ex2_approx(fmaf(__uint_as_float(sr[c]), sl2, -msub));
-                        const float p1 = ex2_approx(fmaf(__uint_as_float(sr[c + 1]), sl2, -msub));
-                        rs0 += p0;
-                        rs1 += p1;
-                        pk[c >> 1] = pack_bf16x2(p0, p1);
+                    for (int e = 0; e < 4; ++e) acc[e] = make_float2(0.f, 0.f);
+#pragma unroll
+                    for (int c = 0; c < 128; c += 8) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float2 xv = __ffma2_rn(make_float2(__uint_as_float(sr[c + 2 * e]),
+                                                                     __uint_as_float(sr[c + 2 * e + 1])), sl2v, nmv);
+                            float2 pr;
+                            if (e >= 4 - EX2_POLY_PER_8 / 2) {
+                                pr = ex2_poly2(xv);
+                            } else {
+                                pr.x = ex2_approx(xv.x);
+                                pr.y = ex2_approx(xv.y);
+                            }
+                            acc[e] = __fadd2_rn(acc[e], pr);
+                            pk[(c >> 1) + e] = pack_bf16x2(pr.x, pr.y);
+                        }
                     }
-                    l += rs0 + rs1;
+                    l += (acc[0].x + acc[0].y) + (acc[1].x + acc[1].y) + ((acc[2].x + acc[2].y) + (acc[3].x + acc[3].y));
                 }
                 tmem_st32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
                 tmem_st32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
