@@ -137,7 +137,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="focus", choices=["focus", "reference"])
     ap.add_argument("--workload", default="M128k")
-    ap.add_argument("--layout", type=int, default=0)
+    ap.add_argument("--layout", type=int, default=1, help="0 = original token order, 1 = class-sorted (group-permuted)")
     ap.add_argument("--ref-rows", type=int, default=2048, help="oracle rows per step (reference arm)")
     ap.add_argument("--cpu-rows", type=int, default=24576, help="oracle rows of the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -177,7 +177,8 @@ def main():
     O = torch.empty_like(Q)
     lse = torch.empty((wl.Hq, wl.n), dtype=torch.float32, device="cuda")
     status = torch.zeros(4, dtype=torch.int32, device="cuda")
-    launches_per_step = 2 + 3 + 1 + (3 if layout == 1 else 0)      # assign x2, build_tiles (3 kernels), attention
+    # assign x2, build_tiles (3 kernels; class-sorted: + 6 per side + ranges + order), attention (+ 3 gathers)
+    launches_per_step = 2 + 3 + 1 + (14 + 3 if layout == 1 else 0)
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
     marks = []

@@ -84,22 +84,29 @@ typedef struct {
     int32_t layout, nqt, nkt, nkw;
     size_t total_bytes;
     size_t counters;   /* uint64[8]: [0] far tile pairs, [1] live far tile pairs, [2] full far tile pairs,
-                                     [3] sorted layout: tile pairs listed in the ranges */
+                                     [3] sorted layout: key tiles listed in the ranges, summed over query blocks,
+                                     [4] sorted layout: non-zero when a head has more than FOCUS_MAX_CLASSES mask values */
     size_t orq, andq;  /* uint32 [B*Hq][nqt]: OR / AND of the member masks of each query tile */
     size_t ork, andk;  /* uint32 [B*Hkv][nkt] */
     size_t gbits;      /* uint32 [B*Hkv][nkt][K][4]: bit j of word j/32 set when key 128*b + j is in group g */
     size_t live;       /* uint32 [B*Hq][nqt][nkw]: bit b set when (a, b) is a far tile pair that may hold a kept pair */
     size_t live_cnt;   /* int32  [B*Hq][nqt]: popcount of the row of `live` */
     /* class-sorted layout only (0 otherwise) */
-    int32_t nqp, nkp;  /* padded sorted lengths (multiples of 256) */
+    int32_t nqp, nkp;  /* capacity of the sorted arrays in rows (multiples of 256): n + room for padding every class segment */
     size_t ncls_q, ncls_k;   /* int32 [B*Hq], [B*Hkv]: distinct mask values of the head */
     size_t cls_q, cls_k;     /* uint32 [heads][FOCUS_MAX_CLASSES]: the mask values, ascending */
-    size_t seg_q, seg_k;     /* int32 [heads][FOCUS_MAX_CLASSES+1]: padded start of each class segment */
-    size_t perm_q, perm_k;   /* int32 [heads][nqp|nkp]: original position of each sorted slot; padding is
-                                -1 on the query side and INT32_MAX on the key side */
-    size_t qrange;           /* int32 [B*Hq][nqp/256][FOCUS_MAX_CLASSES][2]: first and one-past-last sorted
-                                key tile (128 keys) of each key class a 256-row query block must visit */
-    size_t qs, ks, vs;       /* bf16 sorted copies [B*Hq][nqp][D], [B*Hkv][nkp][D] x2 */
+    size_t cnt_q, cnt_k;     /* int32 [heads][FOCUS_MAX_CLASSES]: tokens of each class */
+    size_t seg_q, seg_k;     /* int32 [heads][FOCUS_MAX_CLASSES+1]: first sorted slot of each class segment; query
+                                segments are padded to multiples of 256 slots, key segments to multiples of 128;
+                                entry [ncls] is the number of slots in use */
+    size_t perm_q, perm_k;   /* int32 [heads][nqp|nkp]: original position of each sorted slot, ascending inside a
+                                segment (stable sort); padding is -1 on the query side and INT32_MAX on the key side */
+    size_t qrange;           /* int32 [B*Hq][nqp/256][FOCUS_MAX_CLASSES][2]: first and one-past-last sorted key tile
+                                (128 slots) of each key class that a block of 256 sorted queries must visit */
+    size_t order;            /* int32 [B*Hkv][(Hq/Hkv)*(nqp/256)][2]: (query head, query block) pairs of each KV head
+                                group, most key tiles first */
+    size_t qs, ks, vs;       /* bf16 sorted copies [B*Hq][nqp][D], [B*Hkv][nkp][D] x2, filled by focus_attn_fwd */
+    size_t scratch;          /* build-time scratch (hash sets of mask values, chunk histograms, block costs) */
 } focus_tiles_layout;
 
 /* Library version (major*10000 + minor*100 + patch). */

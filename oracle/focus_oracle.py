@@ -22,6 +22,10 @@ Passages of the paper each function follows:
                         this is the tile-level consequence of Sec. 2 "different-group distant pairs
                         are never computed".
 * ``class_sort``        Sec. 2 "Sort tokens by group (stable sort preserves causal order)".
+* ``sorted_layout``     the padded class-sorted arrays and, per block of sorted queries and key class, the
+                        range of sorted key tiles that can hold an attended pair -- the same Sec. 2 sort
+                        combined with Appendix C's mask (same-class-sharing keys up to the block's last
+                        position; other keys only inside the window).
 
 Parity status: every function above is pinned by the CPU tests.  "parity unpinned": the paper's
 perplexity and benchmark numbers (datasets and trained weights are not available).
@@ -293,3 +297,47 @@ def class_sort(m_h: np.ndarray):
     perm = np.argsort(m_h, kind="stable").astype(np.int64)
     classes, counts = np.unique(m_h, return_counts=True)
     return perm, classes.astype(np.uint32), counts.astype(np.int64)
+
+
+def sorted_layout(mq_h: np.ndarray, mk_h: np.ndarray, window: int, pad_q: int = 256, pad_k: int = 128,
+                  tile: int = 128):
+    """Class-sorted layout of one (query head, KV head) pair, written from its definition.
+
+    Tokens are stably sorted by mask value; each class segment is padded to a multiple of ``pad_q``
+    (queries, padding -1) or ``pad_k`` (keys, padding INT32_MAX).  For every block of ``pad_q`` sorted
+    queries (one class, positions pmin..pmax) and every key class: if the two mask values intersect,
+    the keys of the class with position <= pmax can be attended; otherwise only those with position
+    in [pmin - window, pmax].  The range is given in sorted key tiles of ``tile`` slots,
+    (first, one past last), (0, 0) when empty.
+    Returns dict(cls_q, cnt_q, seg_q, perm_q, cls_k, cnt_k, seg_k, perm_k, ranges [nblk, ncls_k, 2]).
+    """
+    def side(m, pad, fill):
+        perm, cls, cnt = class_sort(m)
+        seg = np.zeros(len(cls) + 1, np.int64)
+        seg[1:] = np.cumsum((cnt + pad - 1) // pad * pad)
+        out = np.full(int(seg[-1]), fill, np.int64)
+        src = 0
+        for c in range(len(cls)):
+            out[seg[c]:seg[c] + cnt[c]] = perm[src:src + cnt[c]]
+            src += cnt[c]
+        return cls, cnt, seg, out
+
+    cls_q, cnt_q, seg_q, perm_q = side(np.asarray(mq_h, np.uint32), pad_q, -1)
+    cls_k, cnt_k, seg_k, perm_k = side(np.asarray(mk_h, np.uint32), pad_k, np.iinfo(np.int32).max)
+    nblk = int(seg_q[-1]) // pad_q
+    ranges = np.zeros((nblk, len(cls_k), 2), np.int64)
+    for blk in range(nblk):
+        rows = perm_q[blk * pad_q:(blk + 1) * pad_q]
+        rows = rows[rows >= 0]
+        jq = int(np.searchsorted(seg_q, blk * pad_q, side="right")) - 1
+        pmin, pmax = int(rows.min()), int(rows.max())
+        for jk in range(len(cls_k)):
+            kp = perm_k[seg_k[jk]:seg_k[jk] + cnt_k[jk]]
+            if int(cls_q[jq]) & int(cls_k[jk]):
+                idx = np.nonzero(kp <= pmax)[0]
+            else:
+                idx = np.nonzero((kp <= pmax) & (kp >= pmin - window))[0]
+            if idx.size:
+                ranges[blk, jk] = ((seg_k[jk] + idx.min()) // tile, (seg_k[jk] + idx.max()) // tile + 1)
+    return dict(cls_q=cls_q, cnt_q=cnt_q, seg_q=seg_q, perm_q=perm_q, cls_k=cls_k, cnt_k=cnt_k, seg_k=seg_k,
+                perm_k=perm_k, ranges=ranges)

@@ -34,8 +34,10 @@ class focus_tiles_layout(C.Structure):
                 ("gbits", C.c_size_t), ("live", C.c_size_t), ("live_cnt", C.c_size_t),
                 ("nqp", C.c_int32), ("nkp", C.c_int32),
                 ("ncls_q", C.c_size_t), ("ncls_k", C.c_size_t), ("cls_q", C.c_size_t), ("cls_k", C.c_size_t),
+                ("cnt_q", C.c_size_t), ("cnt_k", C.c_size_t),
                 ("seg_q", C.c_size_t), ("seg_k", C.c_size_t), ("perm_q", C.c_size_t), ("perm_k", C.c_size_t),
-                ("qrange", C.c_size_t), ("qs", C.c_size_t), ("ks", C.c_size_t), ("vs", C.c_size_t)]
+                ("qrange", C.c_size_t), ("order", C.c_size_t), ("qs", C.c_size_t), ("ks", C.c_size_t),
+                ("vs", C.c_size_t), ("scratch", C.c_size_t)]
 
 
 class FocusError(RuntimeError):

@@ -96,14 +96,18 @@ static int layout_of(const focus_shape* s, int layout, focus_tiles_layout* L) {
         L->ncls_k = take(HK * 4);
         L->cls_q = take(HQ * FOCUS_MAX_CLASSES * 4);
         L->cls_k = take(HK * FOCUS_MAX_CLASSES * 4);
+        L->cnt_q = take(HQ * FOCUS_MAX_CLASSES * 4);
+        L->cnt_k = take(HK * FOCUS_MAX_CLASSES * 4);
         L->seg_q = take(HQ * (FOCUS_MAX_CLASSES + 1) * 4);
         L->seg_k = take(HK * (FOCUS_MAX_CLASSES + 1) * 4);
         L->perm_q = take(HQ * (size_t)L->nqp * 4);
         L->perm_k = take(HK * (size_t)L->nkp * 4);
         L->qrange = take(HQ * (size_t)(L->nqp / 256) * FOCUS_MAX_CLASSES * 2 * 4);
+        L->order = take(HQ * (size_t)(L->nqp / 256) * 2 * 4);
         L->qs = take(HQ * (size_t)L->nqp * s->D * 2);
         L->ks = take(HK * (size_t)L->nkp * s->D * 2);
         L->vs = take(HK * (size_t)L->nkp * s->D * 2);
+        L->scratch = take(sorted_scratch_bytes(s));
     }
     L->total_bytes = off;
     return FOCUS_OK;
@@ -163,6 +167,15 @@ int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, const uint32
     if ((uintptr_t)ws % 256) return fail(FOCUS_ERR_INVALID_ARG, "ws is not 256-byte aligned");
     if (ws_bytes < L.total_bytes)
         return fail(FOCUS_ERR_CAPACITY, "workspace has %zu bytes, %zu needed", ws_bytes, L.total_bytes);
+    if (layout == FOCUS_LAYOUT_CLASS_SORTED) {
+        // masks with exactly topk bits have C(K, topk) values; more than the class table holds is refused here,
+        // other mask patterns with too many values are caught on the device (counters[4], then dev_status)
+        double classes = 1.0;
+        for (int j = 0; j < shape->topk; ++j) classes = classes * (shape->K - j) / (j + 1);
+        if (classes > (double)FOCUS_MAX_CLASSES + 0.5)
+            return fail(FOCUS_ERR_UNSUPPORTED, "class-sorted layout: C(K=%d, topk=%d) mask values exceed %d", shape->K,
+                        shape->topk, FOCUS_MAX_CLASSES);
+    }
     if ((rc = require_sm100())) return rc;
     return launch_build_tiles(shape, mq, mk, layout, L, (char*)ws, (cudaStream_t)stream);
 }

@@ -83,6 +83,17 @@ struct AttnParams {
     float* lse;
     int32_t* status;
     long long nitems;
+    // class-sorted layout: Q/K/V are the sorted copies, tiles are tiles of the sorted order
+    int sorted;
+    int nqp, nkp, nqblk;
+    int ipb;                 // items per block of 256 sorted queries (1, or 2 when an item is one query tile)
+    const int32_t* perm_q;
+    const int32_t* perm_k;
+    const uint32_t* cls_k;
+    const int32_t* ncls_k;
+    const int32_t* qrange;
+    const int32_t* order;
+    const unsigned long long* counters;
 };
 
 // Enumerates the key tiles a 256-row query block visits, in increasing order.  Every role of the
@@ -93,9 +104,22 @@ struct TileWalk {
     int f0, b_last, b, wd;
     uint32_t bits;
     bool far_phase;
+    // class-sorted layout: the ranges of sorted key tiles, key class by key class
+    const int32_t* qr;
+    int nck, jk, rend;
+    bool sorted;
 
     // a0 = first 128-row query tile of the item, nq = number of query tiles of the item (1 or 2)
     __device__ __forceinline__ void init(const AttnParams& p, int hq, int a0, int nq) {
+        sorted = p.sorted != 0;
+        if (sorted) {
+            const int hk = (hq / p.Hq) * p.Hkv + (hq % p.Hq) / p.G;
+            qr = p.qrange + ((size_t)hq * p.nqblk + (a0 >> 1)) * FOCUS_MAX_CLASSES * 2;
+            nck = __ldg(p.ncls_k + hk);
+            jk = -1;
+            b = rend = 0;
+            return;
+        }
         const long long last_row = min((long long)p.n, (long long)(a0 + nq) * 128) - 1;
         b_last = (int)(last_row / 128);
         f0 = 0;
@@ -111,7 +135,16 @@ struct TileWalk {
         bits = 0;
         b = f0;
     }
+    // next key tile, or -1; in the sorted layout `jk` is then the class index of that tile
     __device__ __forceinline__ int next() {
+        if (sorted) {
+            while (b >= rend) {
+                if (++jk >= nck) return -1;
+                b = __ldg(qr + 2 * jk);
+                rend = __ldg(qr + 2 * jk + 1);
+            }
+            return b++;
+        }
         if (far_phase) {
             for (;;) {
                 if (bits) {
@@ -240,6 +273,14 @@ __device__ __forceinline__ bool item_of(const AttnParams& p, int round, Item& t)
     const int g = (int)gridDim.x, c = (int)blockIdx.x;
     t.id = (long long)round * g + ((round & 1) ? g - 1 - c : c);
     if (t.id >= p.nitems) return false;
+    if (p.sorted) {
+        const long long e = t.id / p.ipb;
+        t.hq = __ldg(p.order + 2 * e);
+        t.A = __ldg(p.order + 2 * e + 1) * p.ipb + (int)(t.id % p.ipb);
+        t.bb = t.hq / p.Hq;
+        t.h = t.hq % p.Hq;
+        return true;
+    }
     const int per_group = p.nqb * p.G;
     const int grp = (int)(t.id / per_group);              // batch * Hkv + KV head
     const int rem = (int)(t.id % per_group);
@@ -248,6 +289,42 @@ __device__ __forceinline__ bool item_of(const AttnParams& p, int round, Item& t)
     t.h = (grp % p.Hkv) * p.G + rem % p.G;
     t.hq = t.bb * p.Hq + t.h;
     return true;
+}
+
+// number of entries of the ascending 128-entry array `a` that are <= v (fixed-depth search)
+__device__ __forceinline__ int count_le_128(const int32_t* __restrict__ a, int v) {
+    int lo = 0;
+#pragma unroll
+    for (int step = 64; step >= 1; step >>= 1)
+        if (__ldg(a + lo + step - 1) <= v) lo += step;
+    return lo + (lo == 127 && __ldg(a + 127) <= v ? 1 : 0);
+}
+
+// Tile mask in the class-sorted layout.  The keys of a tile belong to one class and their original
+// positions `kpos` ascend, so a row keeps a contiguous range of columns: those at or before its own
+// position and, unless the classes share a group, not further back than the window.  The decisions
+// "no mask needed" / "nothing attended" are taken per warp from the warp's smallest and largest row
+// position.
+__device__ __forceinline__ void build_tile_mask_sorted(TileMask& tm, int w, const int32_t* __restrict__ kpos, bool share,
+                                                       int pos, int wmin, int wmax) {
+    const int k_first = __ldg(kpos), k_last = __ldg(kpos + 127);
+    tm.all_masked = wmax < 0 || k_first > wmax;
+    const bool need_causal = k_last > wmin;
+    const bool need_window = !share && ((long long)wmax - k_first > w);
+    tm.masked = need_causal || need_window;
+    tm.kw[0] = tm.kw[1] = tm.kw[2] = tm.kw[3] = 0xffffffffu;
+    if (tm.masked && !tm.all_masked) {
+        const int hi = need_causal ? (pos < 0 ? 0 : count_le_128(kpos, pos)) : 128;          // columns < hi are causal
+        const long long edge = (long long)pos - w - 1;
+        const int lo = (need_window && pos >= 0 && edge >= 0) ? count_le_128(kpos, (int)edge) : 0;   // columns >= lo are in the window
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int h = hi - 32 * q, l = lo - 32 * q;
+            const uint32_t below_hi = h >= 32 ? 0xffffffffu : (h <= 0 ? 0u : ((1u << h) - 1u));
+            const uint32_t below_lo = l >= 32 ? 0xffffffffu : (l <= 0 ? 0u : ((1u << l) - 1u));
+            tm.kw[q] = below_hi & ~below_lo;
+        }
+    }
 }
 
 template <int D, bool SOFTCAP>
@@ -263,6 +340,12 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t skv = base + NQ * C::TILE_BYTES;            // ring of K / V tiles
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+    if (p.sorted && __ldg(p.counters + 4) != 0ull) {      // more mask values than the sorted layout holds: refuse
+        if (threadIdx.x == 0 && p.status && atomicCAS(p.status, 0, 2) == 0) {
+            p.status[1] = 1; p.status[2] = 0; p.status[3] = (int)blockIdx.x;
+        }
+        return;
+    }
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&ctl.q_full), 1);
         mbar_init(smem_u32(&ctl.q_empty), 1);
@@ -294,22 +377,26 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         if (lane == 0) {
             prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
             long long nload = 0;
-            int it = 0;
+            int it = 0;                     // items processed (items without key tiles are skipped by every role)
             bool ok = true;
             Item t;
-            for (; ok && item_of(p, it, t); ++it) {
+            for (int round = 0; ok && item_of(p, round, t); ++round) {
                 const int A = t.A, hq = t.hq, b = t.bb, h = t.h, hk = h / p.G;
                 const long long item = t.id;
+                TileWalk walk;
+                walk.init(p, hq, A * NQ, NQ);
+                int kb = walk.next();
+                if (kb < 0) continue;
                 if (it > 0 && !ctl_wait(&ctl.q_empty, (it - 1) & 1, &ctl)) { report_timeout(p, &ctl, 10, (int)item); break; }
                 mbar_arrive_expect_tx(smem_u32(&ctl.q_full), NQ * C::TILE_BYTES);
+                // in the sorted layout the copies are indexed [head of the batch][sorted slot]
+                const int qh = p.sorted ? hq : h, qb = p.sorted ? 0 : b;
+                const int kh = p.sorted ? b * p.Hkv + hk : hk;
                 for (int x = 0; x < NQ; ++x)
                     for (int c = 0; c < C::SUBT; ++c)
                         tma_load_4d(sq + x * C::TILE_BYTES + c * C::SUB_BYTES, &tm_q, smem_u32(&ctl.q_full), c * 64,
-                                    (A * NQ + x) * 128, h, b);
-                TileWalk walk;
-                walk.init(p, hq, A * NQ, NQ);
-                int kb;
-                while (ok && (kb = walk.next()) >= 0) {
+                                    (A * NQ + x) * 128, qh, qb);
+                for (; ok && kb >= 0; kb = walk.next()) {
                     for (int kv = 0; kv < 2; ++kv) {
                         const int slot = (int)(nload % C::NSTAGE);
                         const long long use = nload / C::NSTAGE;
@@ -322,10 +409,11 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         mbar_arrive_expect_tx(bar, C::TILE_BYTES);
                         for (int c = 0; c < C::SUBT; ++c)
                             tma_load_4d(skv + slot * C::TILE_BYTES + c * C::SUB_BYTES, kv ? &tm_v : &tm_k, bar, c * 64,
-                                        kb * 128, hk, b);
+                                        kb * 128, kh, qb);
                         ++nload;
                     }
                 }
+                ++it;
             }
         }
         __syncwarp();
@@ -381,12 +469,13 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 return true;
             };
             Item t;
-            for (; ok && item_of(p, it, t); ++it) {
+            for (int round = 0; ok && item_of(p, round, t); ++round) {
                 const int A = t.A, hq = t.hq;
                 const long long item = t.id;
                 TileWalk walk;
                 walk.init(p, hq, A * NQ, NQ);
                 int cur = walk.next();
+                if (cur < 0) continue;
                 if (!ctl_wait(&ctl.q_full, it & 1, &ctl)) { report_timeout(p, &ctl, 20, (int)item); break; }
                 int slot;
                 if (!wait_kv(slot, 21, (int)item)) break;
@@ -451,6 +540,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     first = false;
                     cur = nxt;
                 }
+                ++it;
             }
         }
         __syncwarp();
@@ -468,25 +558,39 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         int it = 0;
         bool ok = true;
         Item t;
-        for (; ok && item_of(p, it, t); ++it) {
+        for (int round = 0; ok && item_of(p, round, t); ++round) {
             const int A = t.A, hq = t.hq, bb = t.bb, h = t.h;
             const long long item = t.id;
             const int hk = bb * p.Hkv + h / p.G;
             const int a = A * NQ + x;
-            const long long i = (long long)a * 128 + row_in_tile;
-            const bool valid = i < p.n;
+            TileWalk walk;
+            walk.init(p, hq, A * NQ, NQ);
+            int kb = walk.next();
+            if (kb < 0) continue;
+            // the row's position in the sequence: its index, or in the sorted layout the position its slot holds
+            long long i = (long long)a * 128 + row_in_tile;
+            int wmin = 0, wmax = 0;
+            if (p.sorted) {
+                i = __ldg(p.perm_q + (size_t)hq * p.nqp + i);                       // -1 in the padding of a segment
+                wmin = __reduce_min_sync(0xffffffffu, i < 0 ? 0x7fffffff : (int)i);
+                wmax = __reduce_max_sync(0xffffffffu, (int)i);
+            }
+            const bool valid = i >= 0 && i < p.n;
             const uint32_t mi = (valid && !p.dense) ? __ldg(p.mq + (size_t)hq * p.n + i) : 0u;
-            const uint32_t aq = (!p.dense && a < p.nqt) ? __ldg(p.andq + (size_t)hq * p.nqt + a) : 0u;
+            const uint32_t aq = (!p.dense && !p.sorted && a < p.nqt) ? __ldg(p.andq + (size_t)hq * p.nqt + a) : 0u;
             const long long dfar = (long long)a * 128 - p.w;
             const int f_x = (!p.dense && dfar > 0) ? (int)(dfar / 128) : 0;   // tiles b < f_x are far for this query tile
             float m_used = -INFINITY, l = 0.f;
-            TileWalk walk;
-            walk.init(p, hq, A * NQ, NQ);
-            int kb;
             bool first = true;
-            while ((kb = walk.next()) >= 0) {
+            for (; kb >= 0; kb = walk.next()) {
                 TileMask tm;
-                build_tile_mask(tm, p, a, kb, i, mi, aq, f_x, hk);
+                if (p.sorted) {
+                    const bool share = (mi & __ldg(p.cls_k + (size_t)hk * FOCUS_MAX_CLASSES + walk.jk)) != 0u;
+                    build_tile_mask_sorted(tm, p.w, p.perm_k + (size_t)hk * p.nkp + (size_t)kb * 128, share,
+                                           valid ? (int)i : -1, wmin, wmax);
+                } else {
+                    build_tile_mask(tm, p, a, kb, i, mi, aq, f_x, hk);
+                }
                 // ---- wait for S
                 const int buf = NQ == 2 ? x : (int)(ns & 1);
                 const uint32_t par = NQ == 2 ? (ns & 1) : ((ns >> 1) & 1);
@@ -608,6 +712,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
             if (valid) p.lse[(size_t)hq * p.n + i] = (m_used + lg2_approx(l)) * LN2;
             tc_fence_before();
+            ++it;
         }
     }
     // ---------------------------------------------------------------------- teardown
@@ -621,9 +726,25 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
     using C = AttnCfg<D>;
     CUtensorMap tq, tk, tv;
     int rc;
-    if ((rc = make_tmap_qkv(&tq, a.q, a.s.batch, a.s.Hq, a.s.n, D))) return rc;
-    if ((rc = make_tmap_qkv(&tk, a.k, a.s.batch, a.s.Hkv, a.s.n, D))) return rc;
-    if ((rc = make_tmap_qkv(&tv, a.v, a.s.batch, a.s.Hkv, a.s.n, D))) return rc;
+    const bool sorted = a.ws && a.L.layout == FOCUS_LAYOUT_CLASS_SORTED;
+    if (sorted) {
+        // gather Q, K, V into the sorted order kept in the workspace; the kernel reads the copies
+        char* ws = const_cast<char*>(a.ws);
+        if ((rc = launch_gather_sorted(&a.s, a.q, a.s.Hq, true, a.L, a.ws, ws + a.L.qs, st))) return rc;
+        if ((rc = launch_gather_sorted(&a.s, a.k, a.s.Hkv, false, a.L, a.ws, ws + a.L.ks, st))) return rc;
+        if ((rc = launch_gather_sorted(&a.s, a.v, a.s.Hkv, false, a.L, a.ws, ws + a.L.vs, st))) return rc;
+        const int HQ = a.s.batch * a.s.Hq, HK = a.s.batch * a.s.Hkv;
+        const focus_tensor sq_t{ws + a.L.qs, (int64_t)HQ * a.L.nqp * D, (int64_t)a.L.nqp * D, D};
+        const focus_tensor sk_t{ws + a.L.ks, (int64_t)HK * a.L.nkp * D, (int64_t)a.L.nkp * D, D};
+        const focus_tensor sv_t{ws + a.L.vs, (int64_t)HK * a.L.nkp * D, (int64_t)a.L.nkp * D, D};
+        if ((rc = make_tmap_qkv(&tq, sq_t, 1, HQ, a.L.nqp, D))) return rc;
+        if ((rc = make_tmap_qkv(&tk, sk_t, 1, HK, a.L.nkp, D))) return rc;
+        if ((rc = make_tmap_qkv(&tv, sv_t, 1, HK, a.L.nkp, D))) return rc;
+    } else {
+        if ((rc = make_tmap_qkv(&tq, a.q, a.s.batch, a.s.Hq, a.s.n, D))) return rc;
+        if ((rc = make_tmap_qkv(&tk, a.k, a.s.batch, a.s.Hkv, a.s.n, D))) return rc;
+        if ((rc = make_tmap_qkv(&tv, a.v, a.s.batch, a.s.Hkv, a.s.n, D))) return rc;
+    }
     AttnParams p;
     p.B = a.s.batch; p.Hq = a.s.Hq; p.Hkv = a.s.Hkv; p.G = a.s.Hq / a.s.Hkv; p.n = a.s.n; p.w = a.s.window; p.K = a.s.K;
     p.nqb = cdiv(a.s.n, 128 * C::NQ);
@@ -640,6 +761,17 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
     p.lse = a.lse;
     p.status = a.dev_status;
     p.nitems = (long long)a.s.batch * a.s.Hq * p.nqb;
+    p.sorted = sorted ? 1 : 0;
+    p.nqp = a.L.nqp; p.nkp = a.L.nkp; p.nqblk = a.L.nqp / 256;
+    p.ipb = 2 / C::NQ;
+    p.perm_q = sorted ? reinterpret_cast<const int32_t*>(a.ws + a.L.perm_q) : nullptr;
+    p.perm_k = sorted ? reinterpret_cast<const int32_t*>(a.ws + a.L.perm_k) : nullptr;
+    p.cls_k = sorted ? reinterpret_cast<const uint32_t*>(a.ws + a.L.cls_k) : nullptr;
+    p.ncls_k = sorted ? reinterpret_cast<const int32_t*>(a.ws + a.L.ncls_k) : nullptr;
+    p.qrange = sorted ? reinterpret_cast<const int32_t*>(a.ws + a.L.qrange) : nullptr;
+    p.order = sorted ? reinterpret_cast<const int32_t*>(a.ws + a.L.order) : nullptr;
+    p.counters = a.ws ? reinterpret_cast<const unsigned long long*>(a.ws + a.L.counters) : nullptr;
+    if (sorted) p.nitems = (long long)a.s.batch * a.s.Hq * p.nqblk * p.ipb;
     int dev = 0, sms = 0;
     if ((rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice"))) return rc;
     if ((rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "cudaDeviceGetAttribute"))) return rc;
@@ -653,8 +785,6 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
 }
 
 int launch_attn_sm100(const AttnArgs& a, cudaStream_t st) {
-    if (a.ws && a.L.layout == FOCUS_LAYOUT_CLASS_SORTED)
-        return fail(FOCUS_ERR_UNSUPPORTED, "class-sorted layout is not available in the tensor-core kernel yet");
     const bool cap = a.s.softcap > 0.f;
     switch (a.s.D) {
         case 64: return cap ? launch_attn_t<64, true>(a, st) : launch_attn_t<64, false>(a, st);

@@ -29,11 +29,25 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // layout-1 padded sorted length: room for every class segment to be rounded up to 256 slots
 inline int sorted_capacity(int n) { return (int)align_up((size_t)n + (size_t)FOCUS_MAX_CLASSES * 255, 256); }
 
+// class-sorted layout, build-time scratch: per head a hash set of mask values (256 x 8 bytes), per head and
+// chunk of 1024 tokens a histogram over classes, and per query block its number of key tiles
+constexpr int SORT_CHUNK = 1024;
+constexpr int SORT_HASH = 256;
+inline size_t sorted_scratch_bytes(const focus_shape* s) {
+    const size_t heads = (size_t)s->batch * (s->Hq + s->Hkv);
+    const size_t nchunk = (size_t)cdiv(s->n, SORT_CHUNK);
+    return align_up(heads * SORT_HASH * 8, 256) + align_up(heads * nchunk * FOCUS_MAX_CLASSES * 4, 256) +
+           align_up((size_t)s->batch * s->Hq * (size_t)(sorted_capacity(s->n) / 256) * 4, 256);
+}
+
 // launchers implemented in the other translation units
 int launch_assign(const focus_shape* s, const focus_tensor& x, int H, const float* centroids, uint32_t* masks,
                   unsigned long long* near_ties, float eps, cudaStream_t st);
 int launch_build_tiles(const focus_shape* s, const uint32_t* mq, const uint32_t* mk, int layout,
                        const focus_tiles_layout& L, char* ws, cudaStream_t st);
+// class-sorted layout: copy the rows of t into the sorted order of the workspace (query or key side)
+int launch_gather_sorted(const focus_shape* s, const focus_tensor& t, int H, bool query, const focus_tiles_layout& L,
+                         const char* ws, char* dst, cudaStream_t st);
 int launch_count_kept(const focus_shape* s, const uint32_t* mq, const focus_tiles_layout& L, const char* ws,
                       unsigned long long* out, cudaStream_t st);
 

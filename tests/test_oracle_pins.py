@@ -360,3 +360,41 @@ def test_class_sort_is_stable_and_preserves_kept_sets():
     share = (mq[pq][:, None] & mk[pk][None, :]) != 0
     Ms = (posk <= posq) & (((posq - posk) <= w) | share)
     assert np.array_equal(Ms, M[np.ix_(pq, pk)])
+
+
+@pytest.mark.parametrize("n,K,t,w", [(700, 4, 2, 40), (1500, 4, 1, 100), (900, 8, 2, 0), (600, 2, 1, 1000)])
+def test_sorted_layout_ranges_cover_exactly_the_tiles_with_kept_pairs(n, K, t, w):
+    """every kept pair of the explicit mask lies in a listed tile of its key class; the first and last listed
+    tile of a sharing class hold a kept pair; listed tiles of a non-sharing class touch the window span"""
+    rng = np.random.default_rng(n + K)
+    mq = np.array([sum(1 << int(g) for g in rng.choice(K, t, replace=False)) for _ in range(n)], np.uint32)
+    mk = np.array([sum(1 << int(g) for g in rng.choice(K, t, replace=False)) for _ in range(n)], np.uint32)
+    L = fo.sorted_layout(mq, mk, w)
+    kept = fo.kept_matrix(mq, mk, w)
+    # permutations are stable class sorts
+    for perm, cls, cnt, seg, m in ((L["perm_q"], L["cls_q"], L["cnt_q"], L["seg_q"], mq),
+                                   (L["perm_k"], L["cls_k"], L["cnt_k"], L["seg_k"], mk)):
+        real = perm[(perm >= 0) & (perm < n)]
+        assert sorted(real.tolist()) == list(range(n))
+        for c in range(len(cls)):
+            part = perm[seg[c]:seg[c] + cnt[c]]
+            assert (m[part] == cls[c]).all() and (np.diff(part) > 0).all()
+    slot_of_key = np.empty(n, np.int64)
+    valid_k = np.nonzero(L["perm_k"] < n)[0]
+    slot_of_key[L["perm_k"][valid_k]] = valid_k
+    cls_of_tile = np.searchsorted(L["seg_k"], np.arange(len(L["perm_k"]) // 128) * 128, side="right") - 1
+    for blk in range(L["ranges"].shape[0]):
+        rows = L["perm_q"][blk * 256:(blk + 1) * 256]
+        rows = rows[rows >= 0]
+        keys = np.nonzero(kept[rows].any(axis=0))[0]
+        tiles = np.unique(slot_of_key[keys] // 128)
+        for tl in tiles:
+            first, last = L["ranges"][blk, cls_of_tile[tl]]
+            assert first <= tl < last
+        jq = int(np.searchsorted(L["seg_q"], blk * 256, side="right")) - 1
+        for jk in range(len(L["cls_k"])):
+            first, last = L["ranges"][blk, jk]
+            if last > first and int(L["cls_q"][jq]) & int(L["cls_k"][jk]):
+                assert first in tiles and last - 1 in tiles
+            if last > first:
+                assert first * 128 >= L["seg_k"][jk] and last * 128 <= L["seg_k"][jk + 1]
