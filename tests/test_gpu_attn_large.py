@@ -35,6 +35,13 @@ def run_sampled(name, per_head, layout=0, dense_too=False):
     return stats, frac
 
 
+@pytest.mark.parametrize("name,per_head,lo,hi", [("cfg3", 48, 0.3, 0.9), ("cfg4", 48, 0.30, 0.40), ("M128k", 64, 0.82, 0.86),
+                                                 ("cfg5", 256, 0.82, 0.85)])
+def test_class_sorted_layout_on_the_large_configs(name, per_head, lo, hi):
+    stats, frac = run_sampled(name, per_head, layout=1)
+    assert lo < frac < hi
+
+
 def test_cfg3_clustered_skewed_groups():
     stats, frac = run_sampled("cfg3", 64, dense_too=True)
     assert 0.3 < frac < 0.9
