@@ -307,6 +307,12 @@ def main():
                           frac_of_burst=attn_tf / peaks["burst"], frac_of_datasheet_2250=attn_tf / 2250.0,
                           flops_per_launch=kept_flop, ms_per_launch=t_attn),
             cpu_baseline=cpu_baseline,
+            other_kernels=dict(
+                focus_assign=dict(bound="hbm", achieved=(wl.Hq + wl.Hkv) * wl.n * (2 * wl.D + 4) / (t_assign * 1e-3) / 1e9,
+                                  peak=peaks["hbm_gbs"], unit="GB/s",
+                                  frac=(wl.Hq + wl.Hkv) * wl.n * (2 * wl.D + 4) / (t_assign * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                  note="two launches (Q heads, K heads); bytes = (2 D + 4) per head vector"),
+                focus_build_tiles=dict(ms=t_tiles, note="integer passes over the masks; launch-latency bound at this size")),
             breakdown=dict(assign_ms=t_assign, build_tiles_ms=t_tiles, attn_ms=t_attn, dense_attn_ms=dense_ms,
                            speedup_vs_dense=dense_ms / t_attn, dense_tflops=dense_flop / (dense_ms * 1e-3) / 1e12,
                            kept_pairs=kept, kept_fraction=kept / wl.dense_pairs(), far_tiles=counters[0],
