@@ -130,6 +130,58 @@ def run_reference(args, wl):
     print(json.dumps(line), flush=True)
 
 
+def run_sweep(args):
+    """--sweep: context-length sweep in the shape of the paper's speedup table (Sec. 3.6 / Table 6): Llama-3-8B-shaped
+    layer (32/8 heads, D=128, w=2048), n = 1K ... 1M, K in {4, 8}, top-k in {1, 2}; per point the same kernel in
+    dense-causal mode, the original layout and the class-sorted layout (gathers included), one JSON line each."""
+    from paper_2604_03260_b200 import binding as fb
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, reps):
+        ts = []
+        for i in range(reps + 1):
+            a, b = ev(), ev()
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            if i > 0 or reps == 1:
+                ts.append(a.elapsed_time(b))
+        return float(np.median(ts))
+
+    lengths = [int(x) for x in args.sweep_n.split(",")]
+    for K, topk in ((4, 1), (4, 2), (8, 1), (8, 2)):
+        for n in lengths:
+            wl = fi.Workload(f"sweep-K{K}-t{topk}-n{n}", 32, 8, 128, n, K, topk, 2048, seed=2000 + K * 10 + topk)
+            shape = fb.shape_of(wl)
+            Q, Kt, V, C = fi.make_inputs(wl, "cuda")
+            mq = torch.empty((wl.Hq, n), dtype=torch.int32, device="cuda")
+            mk = torch.empty((wl.Hkv, n), dtype=torch.int32, device="cuda")
+            fb.focus_assign(shape, Q, wl.Hq, C, mq); fb.focus_assign(shape, Kt, wl.Hkv, C, mk)
+            O = torch.empty_like(Q)
+            lse = torch.empty((wl.Hq, n), dtype=torch.float32, device="cuda")
+            status = torch.zeros(4, dtype=torch.int32, device="cuda")
+            reps = 3 if n <= 262144 else 1
+            row = dict(sweep=True, n=n, K=K, topk=topk, window=wl.window, Hq=32, Hkv=8, D=128)
+            row["dense_ms"] = timed(lambda: fb.focus_attn_fwd(shape, Q, Kt, V, None, None, None, 0, O, lse, status), reps)
+            for layout, name in ((0, "original"), (1, "sorted")):
+                ws = fb.alloc_workspace(shape, layout)
+                row[f"tiles_{name}_ms"] = timed(lambda: fb.focus_build_tiles(shape, mq, mk, layout, ws), reps)
+                row[f"{name}_ms"] = timed(lambda: fb.focus_attn_fwd(shape, Q, Kt, V, mq, mk, ws, layout, O, lse, status), reps)
+                if layout == 0:
+                    cnt = torch.zeros(wl.Hq, dtype=torch.int64, device="cuda")
+                    fb.focus_count_kept(shape, mq, ws, cnt)
+                    torch.cuda.synchronize()
+                    row["kept_fraction"] = cnt.sum().item() / wl.dense_pairs()
+                del ws
+            assert status[0].item() == 0, status.tolist()
+            best = min(row["original_ms"] + row["tiles_original_ms"], row["sorted_ms"] + row["tiles_sorted_ms"])
+            row["speedup_vs_dense"] = row["dense_ms"] / best
+            row["kept_tflops_best"] = 4.0 * wl.D * row["kept_fraction"] * wl.dense_pairs() / (best * 1e-3) / 1e12
+            print(json.dumps(row), flush=True)
+            del Q, Kt, V, O, lse, mq, mk
+            torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -142,7 +194,11 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=24576, help="oracle rows of the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="context-length sweep (one JSON line per point) instead of the bench line")
+    ap.add_argument("--sweep-n", default="1024,2048,4096,8192,16384,32768,65536,131072,262144,524288,1048576")
     args = ap.parse_args()
+    if args.sweep:
+        return run_sweep(args)
     name = args.workload
     wl = fi.WORKLOADS[name.split("@")[0]]
     if "@" in name:
