@@ -9,6 +9,11 @@ Passages of the paper each function follows:
 
 * ``assign``            Sec. 2 "Learned grouping" (Eq. 1) + the top-k membership rule of Sec. 2
                         "Efficiency at inference" and Sec. 3.6.
+* ``assign_hidden``     Sec. 2 "Learned grouping", Eq. 1 as the paper states it: one routing vector per token,
+                        ``W_g h_i`` in d_g dimensions, scored against ``C`` by dot product; top-k of the scores
+                        (row-softmax and the temperature do not change a row's ranking).  The optional per-group
+                        bias is what Sinkhorn's column scaling leaves behind at inference: the balanced
+                        assignment is diag(r) exp(S/tau) diag(c), whose row ranking is that of S + tau log c.
 * ``attn_rows``         Sec. 2 (exact softmax over attended pairs) + Appendix C, first equation
                         (the hard Focus mask), with "same group" read as "membership sets intersect".
 * ``dense_brute``       the O(n^2) masked reference the paper verifies against (Appendix C,
@@ -341,3 +346,26 @@ def sorted_layout(mq_h: np.ndarray, mk_h: np.ndarray, window: int, pad_q: int = 
                 ranges[blk, jk] = ((seg_k[jk] + idx.min()) // tile, (seg_k[jk] + idx.max()) // tile + 1)
     return dict(cls_q=cls_q, cnt_q=cnt_q, seg_q=seg_q, perm_q=perm_q, cls_k=cls_k, cnt_k=cnt_k, seg_k=seg_k,
                 perm_k=perm_k, ranges=ranges)
+
+
+def assign_hidden(h_bits: np.ndarray, Wg: np.ndarray, C: np.ndarray, topk: int, bias=None):
+    """The paper's router.  h_bits uint16 [n, d] (bf16 hidden states), Wg [d, d_g], C [K, d_g], bias [K] or None.
+
+    score[i, g] = <Wg^T h_i, C_g> (+ bias_g), in fp64, in the paper's order (project, then score).  The
+    token joins its ``topk`` best groups; exact ties go to the lower group index.
+    Returns (masks uint32 [n], margins f64 [n]) with margin = score of the topk-th minus the (topk+1)-th
+    group (+inf when topk = K).
+    """
+    H = bf16_bits_to_f64(np.asarray(h_bits))
+    Z = H @ np.asarray(Wg, np.float64)
+    S = Z @ np.asarray(C, np.float64).T
+    if bias is not None:
+        S = S + np.asarray(bias, np.float64)[None, :]
+    n, K = S.shape
+    order = np.lexsort((np.broadcast_to(np.arange(K), S.shape), -S), axis=1)       # score descending, index ascending
+    masks = np.zeros(n, np.uint32)
+    for r in range(topk):
+        masks |= (np.uint32(1) << order[:, r].astype(np.uint32))
+    srt = np.take_along_axis(S, order, axis=1)
+    margins = srt[:, topk - 1] - srt[:, topk] if topk < K else np.full(n, np.inf)
+    return masks, margins

@@ -398,3 +398,59 @@ def test_sorted_layout_ranges_cover_exactly_the_tiles_with_kept_pairs(n, K, t, w
                 assert first in tiles and last - 1 in tiles
             if last > first:
                 assert first * 128 >= L["seg_k"][jk] and last * 128 <= L["seg_k"][jk + 1]
+
+
+def _bf16_bits(x):
+    return torch.from_numpy(np.asarray(x, np.float32)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+
+
+def test_assign_hidden_matches_torch_topk_and_reduces_to_cosine_assign():
+    rng = np.random.default_rng(5)
+    n, d, dg, K, t = 400, 96, 16, 6, 2
+    hb = _bf16_bits(rng.standard_normal((n, d)))
+    W = rng.standard_normal((d, dg)); C = rng.standard_normal((K, dg)); b = rng.standard_normal(K)
+    masks, margins = fo.assign_hidden(hb, W, C, t, bias=b)
+    H = torch.from_numpy(hb.view(np.int16)).view(torch.bfloat16).double()
+    S = (H @ torch.from_numpy(W)) @ torch.from_numpy(C).T + torch.from_numpy(b)
+    idx = torch.topk(S, t, dim=1).indices.numpy()
+    ref = np.zeros(n, np.uint32)
+    for r in range(t):
+        ref |= np.uint32(1) << idx[:, r].astype(np.uint32)
+    assert np.array_equal(masks, ref) and (margins > 0).all()
+    # W = identity, unit centroids, no bias: the ranking of dot products is the ranking of cosines
+    Cn = rng.standard_normal((K, d)); Cn /= np.linalg.norm(Cn, axis=1, keepdims=True)
+    m_hidden, _ = fo.assign_hidden(hb, np.eye(d), Cn, t)
+    m_cos, _ = fo.assign(hb[None], Cn[None].astype(np.float32), t)
+    m_hidden32, _ = fo.assign_hidden(hb, np.eye(d), Cn.astype(np.float32), t)
+    assert np.array_equal(m_hidden32, m_cos[0])
+    # ties go to the lower index; a dominant bias always wins
+    m_tie, mg = fo.assign_hidden(hb[:5], np.zeros((d, dg)), C, 2)
+    assert (m_tie == 0b11).all() and (mg == 0).all()
+    m_bias, _ = fo.assign_hidden(hb, W, C, 1, bias=np.array([0, 0, 0, 1e9, 0, 0.0]))
+    assert (m_bias == 1 << 3).all()
+
+
+def test_bias_is_the_inference_residue_of_sinkhorn_column_scaling():
+    """Sec. 2: Q <- exp(S/tau); N times: divide by the sum over tokens, then by the sum over groups.  The result is
+    diag(r) exp(S/tau) diag(c), so every row ranks its groups like S + tau log c: with bias = tau log c the router
+    reproduces the balanced assignment's top-k."""
+    rng = np.random.default_rng(9)
+    n, d, dg, K, tau = 300, 64, 16, 4, 0.7
+    hb = _bf16_bits(rng.standard_normal((n, d)))
+    W = rng.standard_normal((d, dg)) * 0.2; C = rng.standard_normal((K, dg)); C[0] += 1.5      # group 0 would dominate
+    S = (fo.bf16_bits_to_f64(hb) @ W) @ C.T
+    Q = np.exp(S / tau)
+    logc = np.zeros(K)
+    for _ in range(10):
+        col = Q.sum(axis=0, keepdims=True)
+        Q = Q / col; logc -= np.log(col[0])
+        Q = Q / Q.sum(axis=1, keepdims=True)
+    top_sinkhorn = np.argsort(-Q, axis=1, kind="stable")[:, :2]
+    want = (np.uint32(1) << top_sinkhorn[:, 0].astype(np.uint32)) | (np.uint32(1) << top_sinkhorn[:, 1].astype(np.uint32))
+    got, _ = fo.assign_hidden(hb, W, C, 2, bias=tau * logc)
+    assert np.array_equal(got, want)
+    plain, _ = fo.assign_hidden(hb, W, C, 2)
+    assert (plain != want).any()            # without the bias the unbalanced ranking differs
+    mass = Q.sum(axis=0)                     # Sinkhorn did balance the groups' mass; the plain row softmax does not
+    P = np.exp(S / tau); P /= P.sum(axis=1, keepdims=True)
+    assert mass.max() / mass.min() < 1.05 < P.sum(axis=0).max() / P.sum(axis=0).min()
