@@ -132,6 +132,29 @@ FOCUS_API int focus_assign(const focus_shape* shape, focus_tensor x, int32_t H, 
                  uint32_t* masks_out, unsigned long long* near_ties, float near_tie_eps, void* stream);
 
 /*
+ * focus_assign_hidden -- the router in the paper's own form (Sec. 2 "Learned grouping", Eq. 1): one routing
+ * vector per token, W_g h_i in d_g dimensions, scored against the centroids C [K, d_g] by dot product; the
+ * token joins its `topk` best groups (Sec. 2 "Efficiency at inference"), ties to the lower group index, and
+ * every head of the layer, in the query role and in the key role, uses that one mask.  The temperature and the
+ * row softmax of Eq. 1 do not change a row's ranking and are not applied.  `bias` (nullable) is added to the
+ * scores: Sinkhorn's balanced assignment is diag(r) exp(S/tau) diag(c), whose row ranking is that of
+ * S + tau log c, so bias_g = tau log c_g carries the balancing into inference.
+ *   shape       batch, Hq, Hkv, n, K, topk are read (D is not used here)
+ *   h           device, bf16 hidden states [batch, n, d_model], last dimension contiguous; 16-byte aligned,
+ *               strides (elements) multiples of 8; d_model a multiple of 8
+ *   Wg          device, fp32 [d_model, d_g] row-major      C   device, fp32 [K, d_g]      bias  device fp32 [K] or NULL
+ *   folded      device scratch, fp32 [K, d_model] (K*d_model*4 bytes, 16-byte aligned): receives W_g C_g, the K
+ *               vectors the hidden states are scored against (each hidden state is then read once)
+ *   mq_out      device uint32 [batch*Hq, n] or NULL     mk_out   device uint32 [batch*Hkv, n] or NULL
+ *   near_ties   device, nullable: incremented by the number of tokens whose margin score(topk-th) - score((topk+1)-th),
+ *               in fp32 and in score units, is below near_tie_eps
+ */
+FOCUS_API int focus_assign_hidden(const focus_shape* shape, const void* h, int64_t stride_b, int64_t stride_n,
+                                  int32_t d_model, int32_t d_g, const float* Wg, const float* C, const float* bias,
+                                  float* folded, uint32_t* mq_out, uint32_t* mk_out, unsigned long long* near_ties,
+                                  float near_tie_eps, void* stream);
+
+/*
  * focus_tiles_layout_of -- host-only: sizes and offsets of the tiles workspace.
  * focus_tiles_workspace_bytes -- its total_bytes (0 on bad arguments).
  */

@@ -64,6 +64,8 @@ def lib():
         L.focus_last_error.restype = C.c_char_p
         L.focus_assign.restype = C.c_int
         L.focus_assign.argtypes = [SP, focus_tensor, i32, vp, vp, vp, f32, vp]
+        L.focus_assign_hidden.restype = C.c_int
+        L.focus_assign_hidden.argtypes = [SP, vp, C.c_int64, C.c_int64, i32, i32, vp, vp, vp, vp, vp, vp, vp, f32, vp]
         L.focus_tiles_layout_of.restype = C.c_int
         L.focus_tiles_layout_of.argtypes = [SP, i32, C.POINTER(focus_tiles_layout)]
         L.focus_tiles_workspace_bytes.restype = sz
@@ -123,6 +125,14 @@ def focus_version() -> int:
 def focus_assign(shape, x, H, centroids, masks_out, near_ties=None, near_tie_eps=1e-5, stream=None):
     _check(lib().focus_assign(C.byref(shape), tensor_arg(x), H, _p(centroids), _p(masks_out), _p(near_ties),
                               near_tie_eps, _stream(stream)))
+
+
+def focus_assign_hidden(shape, h, Wg, Cg, bias, folded, mq_out, mk_out, near_ties=None, near_tie_eps=1e-5, stream=None):
+    """h bf16 [batch, n, d_model] (or [n, d_model]); Wg fp32 [d_model, d_g]; Cg fp32 [K, d_g]; folded fp32 [K, d_model] scratch"""
+    assert h.is_cuda and h.dtype == torch.bfloat16 and h.stride(-1) == 1
+    sb, sn = (h.stride(0), h.stride(1)) if h.dim() == 3 else (h.stride(0) * h.shape[0], h.stride(0))
+    _check(lib().focus_assign_hidden(C.byref(shape), _p(h), sb, sn, h.shape[-1], Wg.shape[1], _p(Wg), _p(Cg), _p(bias),
+                                     _p(folded), _p(mq_out), _p(mk_out), _p(near_ties), near_tie_eps, _stream(stream)))
 
 
 def focus_tiles_layout_of(shape, layout) -> focus_tiles_layout:

@@ -158,6 +158,21 @@ int focus_assign(const focus_shape* shape, focus_tensor x, int32_t H, const floa
     return launch_assign(shape, x, H, centroids, masks_out, near_ties, near_tie_eps, (cudaStream_t)stream);
 }
 
+int focus_assign_hidden(const focus_shape* shape, const void* h, int64_t stride_b, int64_t stride_n, int32_t d_model,
+                        int32_t d_g, const float* Wg, const float* C, const float* bias, float* folded, uint32_t* mq_out,
+                        uint32_t* mk_out, unsigned long long* near_ties, float near_tie_eps, void* stream) {
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if (!h || !Wg || !C || !folded) return fail(FOCUS_ERR_INVALID_ARG, "h, Wg, C or folded is NULL");
+    if (!mq_out && !mk_out) return fail(FOCUS_ERR_INVALID_ARG, "mq_out and mk_out are both NULL");
+    if (d_model < 8 || d_model % 8 || d_g < 1) return fail(FOCUS_ERR_INVALID_ARG, "d_model must be a positive multiple of 8 and d_g >= 1");
+    if ((uintptr_t)h % 16 || (uintptr_t)folded % 16 || stride_n % 8 || stride_b % 8 || stride_n < d_model)
+        return fail(FOCUS_ERR_INVALID_ARG, "h and folded must be 16-byte aligned, strides multiples of 8 elements, stride_n >= d_model");
+    if ((rc = require_sm100())) return rc;
+    return launch_assign_hidden(shape, h, stride_b, stride_n, d_model, d_g, Wg, C, bias, folded, mq_out, mk_out, near_ties,
+                                near_tie_eps, (cudaStream_t)stream);
+}
+
 int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, const uint32_t* mk, int32_t layout, void* ws,
                       size_t ws_bytes, void* stream) {
     focus_tiles_layout L;
