@@ -32,6 +32,23 @@ METRIC = "Focus attn-fwd effective TFLOP/s (kept pairs) + speedup vs dense at 12
 UNIT = "TFLOP/s"
 
 
+# DRAM bytes per launch of the attention kernel (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture per
+# entry, see profiles/), keyed by (workload name, layout); only valid for the kernel sources with this digest.
+ATTN_TRAFFIC = {("M-llama3-8b-128k", 1): 5.68e9}
+ATTN_TRAFFIC_SOURCES = "91fa7f96d5bbe61f"
+
+
+def attn_traffic(name, layout):
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("attn_sm100.cu", "sm100_ptx.cuh"):
+        with open(os.path.join(ROOT, "paper_2604_03260_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    if h.hexdigest()[:16] != ATTN_TRAFFIC_SOURCES:
+        return None                      # the kernel changed since the counters were taken
+    return ATTN_TRAFFIC.get((name, layout))
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -358,7 +375,7 @@ def main():
             e2e=e2e,
             gpu_launches=launches_per_step * args.steps,
             roofline=dict(bound="tensor", kernel="focus_attn_kernel", achieved=attn_tf, peak=peaks["sustained"],
-                          unit="TFLOP/s", frac=attn_tf / peaks["sustained"], traffic=None,
+                          unit="TFLOP/s", frac=attn_tf / peaks["sustained"], traffic=attn_traffic(wl.name, layout),
                           peak_source=f"{peaks['source']} bf16 matmul, sustained (kernel timed inside a long step)",
                           frac_of_burst=attn_tf / peaks["burst"], frac_of_datasheet_2250=attn_tf / 2250.0,
                           flops_per_launch=kept_flop, ms_per_launch=t_attn),
