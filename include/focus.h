@@ -201,6 +201,26 @@ FOCUS_API int focus_attn_fwd(const focus_shape* shape, focus_tensor q, focus_ten
                    focus_tensor o, float* lse, int32_t* dev_status, void* stream);
 
 /*
+ * focus_decode_step -- one generation step: the newest token (position n-1, its key and value already appended
+ * to the caches) as the only query, under the same rule as focus_attn_fwd (paper Sec. 2 "Efficiency at inference",
+ * Appendix C first equation): key j is attended iff n-1-j <= window or mq_new[h] & mk[kv(h), j] != 0; exact softmax
+ * over the attended keys, fp32 arithmetic on the bf16 values.  The paper evaluates generation with the method but
+ * gives no procedure; this is the forward rule applied to one row.  Only attended K/V rows are read from HBM.
+ *   shape       n = cached tokens including the new one; Hq / Hkv <= 8
+ *   q, o        device bf16 [batch, Hq, D]: ptr, stride_b, stride_h are used (stride_n ignored)
+ *   k, v        device bf16 caches [batch, Hkv, n, D]; rows 16-byte aligned (ptr 16-byte aligned, strides multiples of 8)
+ *   mq_new      device uint32 [batch*Hq]: membership mask of the new token per query head
+ *   mk          device uint32 [batch*Hkv, n]: membership masks of the cached keys
+ *   lse         device fp32 [batch*Hq], natural log
+ *   ws          device scratch of at least focus_decode_workspace_bytes(shape) bytes, 16-byte aligned (partial results
+ *               of the key splits); contents need not be preserved between calls
+ */
+FOCUS_API size_t focus_decode_workspace_bytes(const focus_shape* shape);
+FOCUS_API int focus_decode_step(const focus_shape* shape, focus_tensor q, focus_tensor k, focus_tensor v,
+                                const uint32_t* mq_new, const uint32_t* mk, focus_tensor o, float* lse, void* ws,
+                                size_t ws_bytes, void* stream);
+
+/*
  * focus_count_kept -- exact number of attended pairs per query head (the denominator-free
  * numerator of "effective FLOP": 4*D flop per attended pair).  Uses the gbits summaries of a
  * workspace built for the same shape and masks (either layout).

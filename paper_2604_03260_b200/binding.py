@@ -75,6 +75,10 @@ def lib():
         L.focus_attn_fwd.restype = C.c_int
         L.focus_attn_fwd.argtypes = [SP, focus_tensor, focus_tensor, focus_tensor, vp, vp, vp, i32, focus_tensor, vp,
                                      vp, vp]
+        L.focus_decode_workspace_bytes.restype = sz
+        L.focus_decode_workspace_bytes.argtypes = [SP]
+        L.focus_decode_step.restype = C.c_int
+        L.focus_decode_step.argtypes = [SP, focus_tensor, focus_tensor, focus_tensor, vp, vp, focus_tensor, vp, vp, sz, vp]
         L.focus_count_kept.restype = C.c_int
         L.focus_count_kept.argtypes = [SP, vp, vp, vp, vp]
         L.focus_count_kept_noalloc.restype = C.c_int
@@ -153,6 +157,21 @@ def focus_build_tiles(shape, mq, mk, layout, ws, stream=None):
 def focus_attn_fwd(shape, q, k, v, mq, mk, tiles_ws, layout, o, lse, dev_status=None, stream=None):
     _check(lib().focus_attn_fwd(C.byref(shape), tensor_arg(q), tensor_arg(k), tensor_arg(v), _p(mq), _p(mk),
                                 _p(tiles_ws), layout, tensor_arg(o), _p(lse), _p(dev_status), _stream(stream)))
+
+
+def focus_decode_workspace_bytes(shape) -> int:
+    return int(lib().focus_decode_workspace_bytes(C.byref(shape)))
+
+
+def focus_decode_step(shape, q, k, v, mq_new, mk, o, lse, ws, stream=None):
+    """q, o bf16 [Hq, D] (or [batch, Hq, D]); k, v bf16 caches [Hkv, n, D]; mq_new int32 [batch*Hq]; mk int32 [batch*Hkv, n]"""
+    def vec_arg(t):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.stride(-1) == 1
+        if t.dim() == 2:
+            return focus_tensor(t.data_ptr(), t.stride(0) * t.shape[0], t.stride(0), t.shape[-1])
+        return focus_tensor(t.data_ptr(), t.stride(0), t.stride(1), t.shape[-1])
+    _check(lib().focus_decode_step(C.byref(shape), vec_arg(q), tensor_arg(k), tensor_arg(v), _p(mq_new), _p(mk), vec_arg(o),
+                                   _p(lse), _p(ws), ws.numel() * ws.element_size(), _stream(stream)))
 
 
 def focus_count_kept(shape, mq, tiles_ws, counts_out, stream=None):

@@ -195,6 +195,25 @@ int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, const uint32
     return launch_build_tiles(shape, mq, mk, layout, L, (char*)ws, (cudaStream_t)stream);
 }
 
+size_t focus_decode_workspace_bytes(const focus_shape* shape) {
+    if (validate_shape(shape)) return 0;
+    return decode_workspace_bytes(shape);
+}
+
+int focus_decode_step(const focus_shape* shape, focus_tensor q, focus_tensor k, focus_tensor v, const uint32_t* mq_new,
+                      const uint32_t* mk, focus_tensor o, float* lse, void* ws, size_t ws_bytes, void* stream) {
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if (!q.ptr || !o.ptr || !mq_new || !mk || !lse || !ws) return fail(FOCUS_ERR_INVALID_ARG, "a pointer argument is NULL");
+    if ((rc = validate_tensor("k", k, true)) || (rc = validate_tensor("v", v, true))) return rc;
+    if ((uintptr_t)ws % 16) return fail(FOCUS_ERR_INVALID_ARG, "ws is not 16-byte aligned");
+    if (ws_bytes < decode_workspace_bytes(shape))
+        return fail(FOCUS_ERR_CAPACITY, "decode workspace has %zu bytes, %zu needed", ws_bytes, decode_workspace_bytes(shape));
+    if ((rc = require_sm100())) return rc;
+    const float scale = shape->scale > 0.f ? shape->scale : 1.0f / sqrtf((float)shape->D);
+    return launch_decode(shape, q, k, v, mq_new, mk, o, lse, (float*)ws, scale, (cudaStream_t)stream);
+}
+
 int focus_count_kept(const focus_shape* shape, const uint32_t* mq, const void* tiles_ws,
                      unsigned long long* counts_out, void* stream) {
     focus_tiles_layout L;

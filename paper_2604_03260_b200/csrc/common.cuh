@@ -46,6 +46,10 @@ int launch_assign(const focus_shape* s, const focus_tensor& x, int H, const floa
 int launch_assign_hidden(const focus_shape* s, const void* h, int64_t sb, int64_t sn, int d, int dg, const float* Wg,
                          const float* C, const float* bias, float* folded, uint32_t* mq, uint32_t* mk,
                          unsigned long long* near_ties, float eps, cudaStream_t st);
+size_t decode_workspace_bytes(const focus_shape* s);
+int launch_decode(const focus_shape* s, const focus_tensor& q, const focus_tensor& k, const focus_tensor& v,
+                  const uint32_t* mq_new, const uint32_t* mk, const focus_tensor& o, float* lse, float* part, float scale,
+                  cudaStream_t st);
 int launch_build_tiles(const focus_shape* s, const uint32_t* mq, const uint32_t* mk, int layout,
                        const focus_tiles_layout& L, char* ws, cudaStream_t st);
 // class-sorted layout: copy the rows of t into the sorted order of the workspace (query or key side)
