@@ -211,6 +211,8 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=24576, help="oracle rows of the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="N > 1: weak = every rank runs the whole workload; strong = the KV heads of one workload are split over the ranks")
     ap.add_argument("--sweep", action="store_true", help="context-length sweep (one JSON line per point) instead of the bench line")
     ap.add_argument("--sweep-n", default="1024,2048,4096,8192,16384,32768,65536,131072,262144,524288,1048576")
     args = ap.parse_args()
@@ -225,24 +227,27 @@ def main():
 
     from paper_2604_03260_b200 import binding as fb      # fails loudly when the library is missing
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2604_03260_b200 import multi
+    rank, world, local = multi.env_world()
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dist = multi.init("nccl", torch.device("cuda", local))
 
     def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
+        multi.barrier(dist)
 
     peaks = load_peaks()
-    shape = fb.shape_of(wl)
     layout = args.layout
     Q, K, V, C = fi.make_inputs(wl, "cuda")
+    wl_full = wl
+    if args.scaling == "strong" and world > 1:
+        # every rank takes a contiguous range of KV heads (with their query heads) of the one workload: no exchange step
+        from dataclasses import replace
+        k0, k1, q0, q1 = multi.head_shard(rank, world, wl.Hq, wl.Hkv)
+        if k1 == k0:
+            raise SystemExit(f"rank {rank}: more ranks than KV heads ({wl.Hkv}); use --scaling weak")
+        Q, K, V, C = Q[q0:q1].contiguous(), K[k0:k1].contiguous(), V[k0:k1].contiguous(), C[k0:k1].contiguous()
+        wl = replace(wl, Hq=q1 - q0, Hkv=k1 - k0)
+    shape = fb.shape_of(wl)
     mq = torch.empty((wl.Hq, wl.n), dtype=torch.int32, device="cuda")
     mk = torch.empty((wl.Hkv, wl.n), dtype=torch.int32, device="cuda")
     near = torch.zeros(1, dtype=torch.int64, device="cuda")
@@ -281,10 +286,7 @@ def main():
     barrier()
     clocks = sampler.stop()
     total_ms = t_start.elapsed_time(t_end)
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = multi.max_over_ranks(total_ms, dist, "cuda")
     assert status[0].item() == 0, f"kernel reported an expired wait: {status.tolist()}"
     ms_step = total_ms / args.steps
     t_assign = float(np.mean([e[0].elapsed_time(e[1]) for e in marks]))
@@ -313,7 +315,9 @@ def main():
             dense_ms.append(a.elapsed_time(b))
     dense_ms = float(np.median(dense_ms))
 
-    value = world * kept_flop / (ms_step * 1e-3) / 1e12
+    # whole-job work: replicas of the workload (weak) or the one workload split by heads (strong)
+    job_flop = world * kept_flop if args.scaling == "weak" else multi.sum_over_ranks(kept_flop, dist, "cuda")
+    value = job_flop / (ms_step * 1e-3) / 1e12
     attn_tf = kept_flop / (t_attn * 1e-3) / 1e12
 
     # end to end through the C ABI with host buffers: H2D of Q, K, V, centroids; D2H of O and lse
@@ -341,11 +345,8 @@ def main():
         b.record()
         barrier()
         e2e_ms = a.elapsed_time(b) / nrep
-        if dist is not None:
-            t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e = dict(value=world * kept_flop / (e2e_ms * 1e-3) / 1e12, unit=UNIT, h2d_bytes_per_step=int(h2d),
+        e2e_ms = multi.max_over_ranks(e2e_ms, dist, "cuda")
+        e2e = dict(value=job_flop / (e2e_ms * 1e-3) / 1e12, unit=UNIT, h2d_bytes_per_step=int(h2d),
                    d2h_bytes_per_step=int(d2h), ms_per_step=e2e_ms)
         del hQ, hK, hV, hO, hL
 
@@ -365,9 +366,12 @@ def main():
     if rank == 0:
         line = dict(
             metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(3, args.warmup),
-            ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+            ms_per_step=ms_step, higher_is_better=True, scaling=args.scaling, vs_baseline=None, dtype="bf16",
             data="synthetic",
-            config=dict(workload=wl.name, Hq=wl.Hq, Hkv=wl.Hkv, D=wl.D, n=wl.n, K=wl.K, topk=wl.topk, window=wl.window,
+            config=dict(workload=wl.name, Hq=wl_full.Hq, Hkv=wl_full.Hkv, D=wl.D, n=wl.n, K=wl.K, topk=wl.topk, window=wl.window,
+                        parallelism=("single GPU" if world == 1 else
+                                     f"{world} replicas, no collective" if args.scaling == "weak" else
+                                     f"KV heads split over {world} ranks, no collective"),
                         softcap=wl.softcap, layout=["original", "class-sorted"][layout],
                         l2="inputs larger than L2 (Q+K+V+O = %.2f GiB); no flush between steps" %
                            ((2 * Q.numel() + 2 * K.numel()) * 2 / 2**30)),
