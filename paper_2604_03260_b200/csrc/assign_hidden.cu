@@ -5,13 +5,13 @@
 // W_g^T h . C_g = h . (W_g C_g), so the projection and the centroids fold into K vectors of length d
 // (a small kernel, once per call); scoring then reads each hidden state exactly once, which makes the
 // pass HBM-bound: 2 d bytes per token.  Thread = token; the block's rows stream through shared
-// memory in chunks of 128 elements (coalesced asynchronous 16-byte copies, two chunks in flight).
+// memory in chunks of 64 elements (coalesced asynchronous 16-byte copies, two chunks in flight).
 #include "common.cuh"
 
 namespace focus {
 
 constexpr int AH_THREADS = 128;      // tokens per block
-constexpr int AH_CHUNK = 128;        // elements of a row per stage
+constexpr int AH_CHUNK = 64;         // elements of a row per stage
 constexpr int AH_ROWB = 2 * AH_CHUNK + 16;   // padded row: conflict-free 16-byte reads per token
 
 // folded[g][e] = sum_j Wg[e][j] * C[g][j]
