@@ -14,8 +14,11 @@
 namespace focus {
 
 constexpr int DEC_KEYS = 128;        // keys per chunk
-constexpr int DEC_THREADS = 256;     // two threads per key for the scores (half of the query heads each), four row
-                                     // quarters x 64 dimension slots for P V
+constexpr int DEC_THREADS = 2 * DEC_KEYS;   // two threads per key for the scores (half of the query heads each);
+                                            // for P V: DEC_ROWGROUPS groups of keys x 64 dimension slots
+constexpr int DEC_NW = DEC_KEYS / 32;       // warps that share one half of the query heads
+constexpr int DEC_ROWGROUPS = DEC_THREADS / 64;
+constexpr int DEC_ROWS_PER_GROUP = DEC_KEYS / DEC_ROWGROUPS;
 constexpr int DEC_GMAX = 8;          // query heads per KV head served by one CTA
 constexpr float DEC_LOG2E = 1.4426950408889634f;
 constexpr float DEC_LN2 = 0.6931471805599453f;
@@ -35,15 +38,15 @@ decode_partial_kernel(const __nv_bfloat16* __restrict__ q, int64_t q_sb, int64_t
     unsigned char* vt = kt + DEC_KEYS * ROWB;                   // [128][ROWB]
     float* qs = reinterpret_cast<float*>(vt + DEC_KEYS * ROWB); // [GMAX][D]
     float* ps = qs + DEC_GMAX * D;                                 // [GMAX][128] probabilities of the chunk
-    float* red = ps + DEC_GMAX * DEC_KEYS;                      // [GMAX][4] per-warp partial maxima / sums
+    float* red = ps + DEC_GMAX * DEC_KEYS;                      // [GMAX][DEC_NW] per-warp partial maxima / sums
     __shared__ __align__(16) uint32_t keep_s[2][DEC_KEYS];      // per key: bit g set when query head g attends it
 
     const int split = blockIdx.x, bh = blockIdx.y;                 // bh = batch * Hkv + KV head
     const int b = bh / Hkv, hk = bh % Hkv;
     const int t = threadIdx.x, lane = t & 31;
     const int key = t & (DEC_KEYS - 1);            // the key of the chunk this thread scores
-    const int gh = t >> 7;                         // ... for the query heads [g_lo, g_hi)
-    const int warp = (t >> 5) & 3;                 // warp index among the four warps that share gh
+    const int gh = t / DEC_KEYS;                   // ... for the query heads [g_lo, g_hi)
+    const int warp = (t >> 5) % DEC_NW;            // warp index among the warps that share gh
     const int GH = (G + 1) / 2;
     const int g_lo = gh * GH, g_hi = min(G, g_lo + GH);
     const int last = n - 1;                                        // position of the new token
@@ -71,12 +74,13 @@ decode_partial_kernel(const __nv_bfloat16* __restrict__ q, int64_t q_sb, int64_t
     const __nv_bfloat16* vb = v + (size_t)b * v_sb + (size_t)hk * v_sh;
     const uint32_t* mkh = mk + (size_t)bh * n;
 
-    // which query heads attend key j
-    auto keep_of = [&](int j) {
+    // mask word of key j (loaded two chunks ahead of its use, so that its latency is never waited for)
+    auto load_mask = [&](int j) { return (j <= last && last - j > w) ? __ldg(mkh + j) : 0u; };
+    // which query heads attend key j, given its mask word
+    auto keep_of = [&](int j, uint32_t mkj) {
         uint32_t keep = 0;
         if (j <= last) {
             const bool local = last - j <= w;
-            const uint32_t mkj = local ? 0u : __ldg(mkh + j);
 #pragma unroll
             for (int g = 0; g < DEC_GMAX; ++g)
                 if (g < G && (local || (mqg[g] & mkj))) keep |= 1u << g;
@@ -101,9 +105,11 @@ decode_partial_kernel(const __nv_bfloat16* __restrict__ q, int64_t q_sb, int64_t
     const int c_end = min(c_begin + chunks_per_split, (n + DEC_KEYS - 1) / DEC_KEYS);
     // Pipeline: K of chunk c+1 is copied while P V of chunk c runs, V of chunk c while its scores are computed.
     uint32_t keep = 0;
+    uint32_t mk_ahead = 0;                         // mask word of this thread's key in the next chunk
     if (c_begin < c_end) {
-        keep = keep_of(c_begin * DEC_KEYS + key);
+        keep = keep_of(c_begin * DEC_KEYS + key, load_mask(c_begin * DEC_KEYS + key));
         keep_s[c_begin & 1][key] = keep;           // both threads of a key write the same word
+        if (c_begin + 1 < c_end) mk_ahead = load_mask((c_begin + 1) * DEC_KEYS + key);
     }
     __syncthreads();
     if (c_begin < c_end) copy_rows(kb, k_sn, kt, c_begin * DEC_KEYS, keep_s[c_begin & 1]);
@@ -113,8 +119,9 @@ decode_partial_kernel(const __nv_bfloat16* __restrict__ q, int64_t q_sb, int64_t
         copy_rows(vb, v_sn, vt, j0, flags);                 // V tile is free: the previous P V ended with a barrier
         uint32_t keep_next = 0;
         if (ch + 1 < c_end) {
-            keep_next = keep_of(j0 + DEC_KEYS + key);
+            keep_next = keep_of(j0 + DEC_KEYS + key, mk_ahead);
             keep_s[(ch + 1) & 1][key] = keep_next;
+            if (ch + 2 < c_end) mk_ahead = load_mask(j0 + 2 * DEC_KEYS + key);
         }
         asm volatile("cp.async.wait_group 1;" ::: "memory");   // K of this chunk has landed
         __syncthreads();
@@ -166,7 +173,7 @@ decode_partial_kernel(const __nv_bfloat16* __restrict__ q, int64_t q_sb, int64_t
                 float mx = s;
 #pragma unroll
                 for (int off = 16; off >= 1; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-                if (lane == 0) red[g * 4 + warp] = mx;
+                if (lane == 0) red[g * DEC_NW + warp] = mx;
             }
         }
         __syncthreads();                        // maxima published; K tile no longer read
@@ -177,7 +184,9 @@ decode_partial_kernel(const __nv_bfloat16* __restrict__ q, int64_t q_sb, int64_t
         for (int g = 0; g < DEC_GMAX; ++g) {
             factor[g] = 1.f; wsum[g] = 0.f;
             if (g < G) {
-                const float cm = fmaxf(fmaxf(red[g * 4], red[g * 4 + 1]), fmaxf(red[g * 4 + 2], red[g * 4 + 3]));
+                float cm = red[g * DEC_NW];
+#pragma unroll
+                for (int ww = 1; ww < DEC_NW; ++ww) cm = fmaxf(cm, red[g * DEC_NW + ww]);
                 const float m_new = fmaxf(m_run[g], cm);
                 factor[g] = (m_run[g] == -INFINITY) ? 0.f : exp2f(m_run[g] - m_new);    // nothing accumulated yet: O and l are 0
                 m_run[g] = m_new;
@@ -194,20 +203,25 @@ decode_partial_kernel(const __nv_bfloat16* __restrict__ q, int64_t q_sb, int64_t
         __syncthreads();                        // maxima consumed by everyone
 #pragma unroll
         for (int g = 0; g < DEC_GMAX; ++g)
-            if (g >= g_lo && g < g_hi && lane == 0) red[g * 4 + warp] = wsum[g];
+            if (g >= g_lo && g < g_hi && lane == 0) red[g * DEC_NW + warp] = wsum[g];
         asm volatile("cp.async.wait_group 1;" ::: "memory");   // V of this chunk has landed
         __syncthreads();
 #pragma unroll
         for (int g = 0; g < DEC_GMAX; ++g)
-            if (g < G) l_run[g] = l_run[g] * factor[g] + (red[g * 4] + red[g * 4 + 1]) + (red[g * 4 + 2] + red[g * 4 + 3]);
-        // ---- P V: 64 threads span the output dimensions, the four quarters of the CTA take 32 keys each
+            if (g < G) {
+                float ssum = red[g * DEC_NW];
+#pragma unroll
+                for (int ww = 1; ww < DEC_NW; ++ww) ssum += red[g * DEC_NW + ww];
+                l_run[g] = l_run[g] * factor[g] + ssum;
+            }
+        // ---- P V: 64 threads span the output dimensions, each group of 64 threads takes its share of the keys
         {
             const int quarter = t >> 6, dp = t & 63;
 #pragma unroll
             for (int g = 0; g < DEC_GMAX; ++g)
 #pragma unroll
                 for (int e = 0; e < DPT; ++e) o_acc[g][e] *= factor[g];
-            for (int r = quarter * 32; r < quarter * 32 + 32; r += 4) {
+            for (int r = quarter * DEC_ROWS_PER_GROUP; r < (quarter + 1) * DEC_ROWS_PER_GROUP; r += 4) {
                 const uint4 kf = *reinterpret_cast<const uint4*>(&flags[r]);
                 if (!(kf.x | kf.y | kf.z | kf.w)) continue;              // uniform across the half: none of the four keys attended
                 float vv[4][DPT];
@@ -244,9 +258,9 @@ decode_partial_kernel(const __nv_bfloat16* __restrict__ q, int64_t q_sb, int64_t
         keep = keep_next;
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    // ---- add the four quarters, then the partial result of this split: [query head][split][2 + D] = (max, sum, O)
+    // ---- add the row groups, then the partial result of this split: [query head][split][2 + D] = (max, sum, O)
     __syncthreads();
-    float* xch = reinterpret_cast<float*>(kt);              // [3][GMAX][D] (the K tile is no longer needed)
+    float* xch = reinterpret_cast<float*>(kt);              // [row groups - 1][GMAX][D] (the K and V tiles are no longer needed)
     const int quarter = t >> 6, dp = t & 63;
     if (quarter > 0) {
 #pragma unroll
@@ -262,9 +276,12 @@ decode_partial_kernel(const __nv_bfloat16* __restrict__ q, int64_t q_sb, int64_t
                 float* dst = part + (((size_t)b * Hq + hk * G + g) * nsplit + split) * (D + 2);
                 if (t == 0) { dst[0] = m_run[g]; dst[1] = l_run[g]; }
 #pragma unroll
-                for (int e = 0; e < DPT; ++e)
-                    dst[2 + dp * DPT + e] = o_acc[g][e] + xch[g * D + dp * DPT + e] + xch[(DEC_GMAX + g) * D + dp * DPT + e] +
-                                            xch[(2 * DEC_GMAX + g) * D + dp * DPT + e];
+                for (int e = 0; e < DPT; ++e) {
+                    float a = o_acc[g][e];
+#pragma unroll
+                    for (int qq = 0; qq < DEC_ROWGROUPS - 1; ++qq) a += xch[(qq * DEC_GMAX + g) * D + dp * DPT + e];
+                    dst[2 + dp * DPT + e] = a;
+                }
             }
         }
     }
@@ -297,10 +314,10 @@ decode_merge_kernel(const float* __restrict__ part, int nsplit, int D, int Hq, _
 static int decode_splits(const focus_shape* s) {
     const int chunks = cdiv(s->n, DEC_KEYS);
     const int heads = s->batch * s->Hkv;
-    int want = cdiv(4 * 148, heads);                 // about four CTAs per SM in total
+    int want = cdiv(4 * 148, heads);                 // about four CTAs per SM in total (two rounds of two resident ones)
     if (want > chunks) want = chunks;
     if (want < 1) want = 1;
-    if (want > 256) want = 256;
+    if (want > 512) want = 512;
     return want;
 }
 
@@ -316,7 +333,7 @@ static int launch_decode_d(const focus_shape* s, const focus_tensor& q, const fo
     const int chunks = cdiv(s->n, DEC_KEYS);
     const int cps = cdiv(chunks, nsplit);
     const size_t smem = (size_t)2 * DEC_KEYS * (2 * D + 16) + (size_t)DEC_GMAX * D * 4 + (size_t)DEC_GMAX * DEC_KEYS * 4 +
-                        (size_t)DEC_GMAX * 4 * 4;
+                        (size_t)DEC_GMAX * DEC_NW * 4;
     auto kern = decode_partial_kernel<D>;
     int rc = check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
                         "cudaFuncSetAttribute(decode)");
