@@ -204,7 +204,7 @@ FOCUS_API int focus_attn_fwd(const focus_shape* shape, focus_tensor q, focus_ten
  * focus_decode_step -- one generation step: the newest token (position n-1, its key and value already appended
  * to the caches) as the only query, under the same rule as focus_attn_fwd (paper Sec. 2 "Efficiency at inference",
  * Appendix C first equation): key j is attended iff n-1-j <= window or mq_new[h] & mk[kv(h), j] != 0; exact softmax
- * over the attended keys, fp32 arithmetic on the bf16 values.  The paper evaluates generation with the method but
+ * over the attended keys; bf16 operands, fp32 accumulation, probabilities rounded to bf16 before P V.  The paper evaluates generation with the method but
  * gives no procedure; this is the forward rule applied to one row.  Only attended K/V rows are read from HBM.
  *   shape       n = cached tokens including the new one; Hq / Hkv <= 8
  *   q, o        device bf16 [batch, Hq, D]: ptr, stride_b, stride_h are used (stride_n ignored)

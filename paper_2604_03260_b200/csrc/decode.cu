@@ -3,319 +3,294 @@
 // the new token at position n-1 attends key j when n-1-j <= w or its groups meet the key's groups.
 // This is the generation use of the method (the paper evaluates generation but gives no procedure).
 //
-// HBM-bound: only the K and V rows of attended keys are read.  Split over the keys: a CTA owns a
-// range of keys of one KV head and serves the G query heads that share it; per chunk of 128 keys the
-// attended rows are copied to shared memory (coalesced asynchronous 16-byte copies, skipped row by
-// row when no query head of the group attends the key), thread = key computes the G scores, thread =
-// output dimension accumulates P V; the partial (max, sum, O) of every split is merged by a second
-// kernel.  fp32 throughout on the exact bf16 values; probabilities are not rounded.
+// HBM-bound: only the K and V rows of attended keys are read, each once per KV head for all the query
+// heads that share it.  The keys are split over CTAs and, inside a CTA, over warps that never synchronise
+// with one another; the partial (max, sum, O) of every warp is merged by a second kernel.  bf16 operands,
+// fp32 accumulation, probabilities rounded to bf16 before P V (as in the forward pass).
 #include "common.cuh"
 
 namespace focus {
 
-constexpr int DEC_KEYS = 128;        // keys per chunk
-constexpr int DEC_THREADS = 2 * DEC_KEYS;   // two threads per key for the scores (half of the query heads each);
-                                            // for P V: DEC_ROWGROUPS groups of keys x 64 dimension slots
-constexpr int DEC_NW = DEC_KEYS / 32;       // warps that share one half of the query heads
-constexpr int DEC_ROWGROUPS = DEC_THREADS / 64;
-constexpr int DEC_ROWS_PER_GROUP = DEC_KEYS / DEC_ROWGROUPS;
-constexpr int DEC_GMAX = 8;          // query heads per KV head served by one CTA
+constexpr int DEC_GMAX = 8;          // query heads per KV head served together (rows of the 16-row MMA tile)
+constexpr int DEC_GK = 16;           // keys per warp step
+constexpr int DEC_NST = 3;           // stages of a warp's private K/V ring
 constexpr float DEC_LOG2E = 1.4426950408889634f;
 constexpr float DEC_LN2 = 0.6931471805599453f;
 
+template <int D> struct DecCfg {
+    static constexpr int WARPS = D == 256 ? 4 : 8;                 // warps per CTA (shared memory bounds it)
+    static constexpr int ROWB = 2 * D + 16;                        // padded row: conflict-free ldmatrix rows
+    static constexpr int STAGE = 2 * DEC_GK * ROWB;                // K rows then V rows of one step
+    static constexpr size_t SMEM = (size_t)WARPS * DEC_NST * STAGE;
+};
+
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                               uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ uint32_t dec_pack_bf16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// Every warp works on its own: steps of 16 keys, a private ring of K/V rows in shared memory filled with
+// asynchronous copies (a row is copied only when some query head of the group attends the key), no
+// CTA-wide barrier in the loop.  The G <= 8 query heads that share the KV head are the rows of a 16-row
+// warp-level MMA tile (a tile of the 5th-generation tensor cores needs 64 rows and would be 7/8 padding):
+// S = Q K^T with K rows as the column operand, P V with V rows through a transposing matrix load.
+// Each warp keeps its own running maximum, sum and O and writes its own partial result.
 template <int D>
-__global__ void __launch_bounds__(DEC_THREADS)
+__global__ void __launch_bounds__(DecCfg<D>::WARPS * 32)
 decode_partial_kernel(const __nv_bfloat16* __restrict__ q, int64_t q_sb, int64_t q_sh, const __nv_bfloat16* __restrict__ k,
                       int64_t k_sb, int64_t k_sh, int64_t k_sn, const __nv_bfloat16* __restrict__ v, int64_t v_sb,
                       int64_t v_sh, int64_t v_sn, const uint32_t* __restrict__ mq_new, const uint32_t* __restrict__ mk,
-                      int Hq, int Hkv, int G, int n, int w, float scale, float softcap, int nsplit, int chunks_per_split,
+                      int Hq, int Hkv, int G, int n, int w, float scale, float softcap, int nsplit, int groups_per_split,
                       float* __restrict__ part) {
-    constexpr int ROWB = 2 * D + 16;                 // padded row: conflict-free 16-byte reads per key
-    constexpr int VEC = D / 8;                       // 16-byte pieces per row
-    constexpr int DPT = D / 64;                      // output dimensions per thread (64 threads span a row)
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    unsigned char* kt = smem_raw;                                  // [128][ROWB]
-    unsigned char* vt = kt + DEC_KEYS * ROWB;                   // [128][ROWB]
-    float* qs = reinterpret_cast<float*>(vt + DEC_KEYS * ROWB); // [GMAX][D]
-    float* ps = qs + DEC_GMAX * D;                                 // [GMAX][128] probabilities of the chunk
-    float* red = ps + DEC_GMAX * DEC_KEYS;                      // [GMAX][DEC_NW] per-warp partial maxima / sums
-    __shared__ __align__(16) uint32_t keep_s[2][DEC_KEYS];      // per key: bit g set when query head g attends it
-
+    using C = DecCfg<D>;
+    constexpr int VEC = D / 8;                                     // 16-byte pieces per row
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ uint32_t kflag_s[C::WARPS][DEC_NST][DEC_GK];        // per staged key: bit g set when query head g attends it
     const int split = blockIdx.x, bh = blockIdx.y;                 // bh = batch * Hkv + KV head
     const int b = bh / Hkv, hk = bh % Hkv;
-    const int t = threadIdx.x, lane = t & 31;
-    const int key = t & (DEC_KEYS - 1);            // the key of the chunk this thread scores
-    const int gh = t / DEC_KEYS;                   // ... for the query heads [g_lo, g_hi)
-    const int warp = (t >> 5) % DEC_NW;            // warp index among the warps that share gh
-    const int GH = (G + 1) / 2;
-    const int g_lo = gh * GH, g_hi = min(G, g_lo + GH);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, qd = lane & 3;                        // this thread's query head (MMA row) and column pair
     const int last = n - 1;                                        // position of the new token
     const float sl2 = (softcap > 0.f ? softcap : scale) * DEC_LOG2E;   // logits in log2 units: sl2 * S or sl2 * tanh(S scale / cap)
     const float cap_in = softcap > 0.f ? scale / softcap : 0.f;
+    unsigned char* ring = smem_raw + (size_t)warp * DEC_NST * C::STAGE;
+    const uint32_t ring_u32 = (uint32_t)__cvta_generic_to_shared(ring);
 
-    for (int i = t; i < G * D; i += DEC_THREADS) {
-        const int g = i / D, d = i % D;
-        qs[i] = __bfloat162float(q[(size_t)b * q_sb + (size_t)(hk * G + g) * q_sh + d]);
-    }
-    // rows that are never copied are still multiplied by probability 0: keep them finite
-    for (int i = t; i < DEC_KEYS * ROWB / 16; i += DEC_THREADS) reinterpret_cast<uint4*>(vt)[i] = make_uint4(0, 0, 0, 0);
-    uint32_t mqg[DEC_GMAX];
-#pragma unroll
-    for (int g = 0; g < DEC_GMAX; ++g) mqg[g] = g < G ? __ldg(mq_new + (size_t)b * Hq + hk * G + g) : 0u;
+    // rows that are never copied still enter the MMAs (with probability 0): keep them finite
+    for (int i = lane; i < DEC_NST * C::STAGE / 16; i += 32) reinterpret_cast<uint4*>(ring)[i] = make_uint4(0, 0, 0, 0);
+    __syncwarp();
 
-    float m_run[DEC_GMAX], l_run[DEC_GMAX], o_acc[DEC_GMAX][DPT];
+    // Q as the row operand: rows >= G and rows 8..15 are zero
+    uint32_t qa[D / 16][2];
+    {
+        const __nv_bfloat16* qrow = q + (size_t)b * q_sb + (size_t)(hk * G + (g < G ? g : 0)) * q_sh;
 #pragma unroll
-    for (int g = 0; g < DEC_GMAX; ++g) {
-        m_run[g] = -INFINITY; l_run[g] = 0.f;
-#pragma unroll
-        for (int e = 0; e < DPT; ++e) o_acc[g][e] = 0.f;
+        for (int ks = 0; ks < D / 16; ++ks) {
+            qa[ks][0] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd * 2) : 0u;
+            qa[ks][1] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + qd * 2) : 0u;
+        }
     }
+    uint32_t mq_all[DEC_GMAX];                                     // every lane needs all heads' masks to flag its key
+#pragma unroll
+    for (int gg = 0; gg < DEC_GMAX; ++gg) mq_all[gg] = gg < G ? __ldg(mq_new + (size_t)b * Hq + hk * G + gg) : 0u;
+
     const __nv_bfloat16* kb = k + (size_t)b * k_sb + (size_t)hk * k_sh;
     const __nv_bfloat16* vb = v + (size_t)b * v_sb + (size_t)hk * v_sh;
     const uint32_t* mkh = mk + (size_t)bh * n;
 
-    // mask word of key j (loaded two chunks ahead of its use, so that its latency is never waited for)
-    auto load_mask = [&](int j) { return (j <= last && last - j > w) ? __ldg(mkh + j) : 0u; };
-    // which query heads attend key j, given its mask word
-    auto keep_of = [&](int j, uint32_t mkj) {
-        uint32_t keep = 0;
-        if (j <= last) {
-            const bool local = last - j <= w;
-#pragma unroll
-            for (int g = 0; g < DEC_GMAX; ++g)
-                if (g < G && (local || (mqg[g] & mkj))) keep |= 1u << g;
-        }
-        return keep;
+    // this warp's steps: groups g0 + warp, g0 + warp + WARPS, ... of 16 keys
+    const int total_groups = (n + DEC_GK - 1) / DEC_GK;
+    const int g_begin = split * groups_per_split;
+    const int g_end = min(g_begin + groups_per_split, total_groups);
+    const int nsteps = g_begin + warp < g_end ? (g_end - g_begin - warp + C::WARPS - 1) / C::WARPS : 0;
+    auto first_key = [&](int step) { return (g_begin + warp + step * C::WARPS) * DEC_GK; };
+
+    // mask word of the key lane % 16 of a step (0 when it is local or past the end: not needed then)
+    auto load_mask = [&](int step) {
+        const int j = first_key(step) + (lane & 15);
+        return (step < nsteps && j <= last && last - j > w) ? __ldg(mkh + j) : 0u;
     };
-    // copy the attended rows of a chunk: 16 consecutive threads copy one row; one commit group per call
-    auto copy_rows = [&](const __nv_bfloat16* src, int64_t sn, unsigned char* dst, int j0, const uint32_t* flags) {
+    // flag the 16 keys of a step and start copying the attended rows into ring stage `st` (16-byte asynchronous
+    // copies, 16 consecutive lanes per row); one commit group per call, also when nothing is copied
+    auto issue = [&](int step, int st, uint32_t mkj) {
+        if (step < nsteps) {
+            uint32_t bits = 0;
+            const int j0 = first_key(step);
+            const int j = j0 + (lane & 15);
+            if (j <= last) {
+                const bool local = last - j <= w;
 #pragma unroll
-        for (int i = 0; i < VEC / 2; ++i) {
-            const int qd = i * DEC_THREADS + t;
-            const int r = qd / VEC, c = qd % VEC;
-            if (flags[r]) {
-                const uint32_t da = (uint32_t)__cvta_generic_to_shared(dst + r * ROWB + c * 16);
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(da), "l"(src + (size_t)(j0 + r) * sn + c * 8) : "memory");
+                for (int gg = 0; gg < DEC_GMAX; ++gg)
+                    if (gg < G && (local || (mq_all[gg] & mkj))) bits |= 1u << gg;
+            }
+            if (lane < DEC_GK) kflag_s[warp][st][lane] = bits;
+            unsigned char* dst = ring + (size_t)st * C::STAGE;
+#pragma unroll
+            for (int i = 0; i < DEC_GK * VEC / 32; ++i) {
+                const int idx = i * 32 + lane;
+                const int r = idx / VEC, c = idx % VEC;
+                const uint32_t rb = __shfl_sync(0xffffffffu, bits, r);
+                if (rb) {
+                    const uint32_t dk = (uint32_t)__cvta_generic_to_shared(dst + r * C::ROWB + c * 16);
+                    const uint32_t dv = dk + DEC_GK * C::ROWB;
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dk), "l"(kb + (size_t)(j0 + r) * k_sn + c * 8) : "memory");
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dv), "l"(vb + (size_t)(j0 + r) * v_sn + c * 8) : "memory");
+                }
             }
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
 
-    const int c_begin = split * chunks_per_split;
-    const int c_end = min(c_begin + chunks_per_split, (n + DEC_KEYS - 1) / DEC_KEYS);
-    // Pipeline: K of chunk c+1 is copied while P V of chunk c runs, V of chunk c while its scores are computed.
-    uint32_t keep = 0;
-    uint32_t mk_ahead = 0;                         // mask word of this thread's key in the next chunk
-    if (c_begin < c_end) {
-        keep = keep_of(c_begin * DEC_KEYS + key, load_mask(c_begin * DEC_KEYS + key));
-        keep_s[c_begin & 1][key] = keep;           // both threads of a key write the same word
-        if (c_begin + 1 < c_end) mk_ahead = load_mask((c_begin + 1) * DEC_KEYS + key);
-    }
-    __syncthreads();
-    if (c_begin < c_end) copy_rows(kb, k_sn, kt, c_begin * DEC_KEYS, keep_s[c_begin & 1]);
-    for (int ch = c_begin; ch < c_end; ++ch) {
-        const int j0 = ch * DEC_KEYS;
-        const uint32_t* flags = keep_s[ch & 1];
-        copy_rows(vb, v_sn, vt, j0, flags);                 // V tile is free: the previous P V ended with a barrier
-        uint32_t keep_next = 0;
-        if (ch + 1 < c_end) {
-            keep_next = keep_of(j0 + DEC_KEYS + key, mk_ahead);
-            keep_s[(ch + 1) & 1][key] = keep_next;
-            if (ch + 2 < c_end) mk_ahead = load_mask(j0 + 2 * DEC_KEYS + key);
-        }
-        asm volatile("cp.async.wait_group 1;" ::: "memory");   // K of this chunk has landed
-        __syncthreads();
-        // ---- thread = (key, half of the query heads): scores, packed pairs (even dims in .x, odd dims in .y)
-        float sc[DEC_GMAX];
+    float m_run = -INFINITY, l_run = 0.f;          // of head g (the four threads of a quad hold the same values)
+    float o[D / 8][4];
 #pragma unroll
-        for (int g = 0; g < DEC_GMAX; ++g) sc[g] = 0.f;
-        if (keep) {
-            float2 s2[DEC_GMAX / 2 + 1];
+    for (int nt = 0; nt < D / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+
+    // prologue: NST - 1 steps in flight, the mask words of the next one on their way
 #pragma unroll
-            for (int gg = 0; gg < DEC_GMAX / 2 + 1; ++gg) s2[gg] = make_float2(0.f, 0.f);
-            const unsigned char* row = kt + key * ROWB;
-#pragma unroll 4
-            for (int vv = 0; vv < VEC; ++vv) {
-                const uint4 rv = *reinterpret_cast<const uint4*>(row + vv * 16);
-                const uint32_t wds[4] = {rv.x, rv.y, rv.z, rv.w};
-                float2 x[4];
+    for (int st = 0; st < DEC_NST - 1; ++st) issue(st, st, load_mask(st));
+    uint32_t mk_ahead = load_mask(DEC_NST - 1);
+    for (int step = 0; step < nsteps; ++step) {
+        const int st = step % DEC_NST;
+        issue(step + DEC_NST - 1, (step + DEC_NST - 1) % DEC_NST, mk_ahead);     // the stage freed by the previous step
+        mk_ahead = load_mask(step + DEC_NST);
+        asm volatile("cp.async.wait_group %0;" ::"n"(DEC_NST - 1) : "memory");
+        __syncwarp();
+        // ---- flags of this thread's four keys: 2 qd, 2 qd + 1, 8 + 2 qd, 9 + 2 qd
+        const uint2 f01 = *reinterpret_cast<const uint2*>(&kflag_s[warp][st][qd * 2]);
+        const uint2 f23 = *reinterpret_cast<const uint2*>(&kflag_s[warp][st][8 + qd * 2]);
+        const uint32_t any4 = f01.x | f01.y | f23.x | f23.y;
+        if (__any_sync(0xffffffffu, any4 != 0u)) {
+            const uint32_t kst = ring_u32 + st * C::STAGE, vst = kst + DEC_GK * C::ROWB;
+            // ---- S = Q K^T for 16 keys: two 8-key column tiles
+            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+            {
+                const int mi = lane >> 3, mr = lane & 7;           // matrix index and row for the matrix loads
+                const uint32_t kaddr = kst + (mr + 8 * (mi >> 1)) * C::ROWB + 16 * (mi & 1);
 #pragma unroll
-                for (int e = 0; e < 4; ++e) x[e] = make_float2(__uint_as_float(wds[e] << 16), __uint_as_float(wds[e] & 0xffff0000u));
-#pragma unroll
-                for (int gg = 0; gg < DEC_GMAX / 2 + 1; ++gg) {
-                    const int g = g_lo + gg;
-                    if (gg < GH && g < G) {
-                        const float4 a0 = *reinterpret_cast<const float4*>(qs + g * D + vv * 8);
-                        const float4 a1 = *reinterpret_cast<const float4*>(qs + g * D + vv * 8 + 4);
-                        float2 acc = s2[gg];
-                        acc = __ffma2_rn(x[0], make_float2(a0.x, a0.y), acc);
-                        acc = __ffma2_rn(x[1], make_float2(a0.z, a0.w), acc);
-                        acc = __ffma2_rn(x[2], make_float2(a1.x, a1.y), acc);
-                        acc = __ffma2_rn(x[3], make_float2(a1.z, a1.w), acc);
-                        s2[gg] = acc;
-                    }
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    uint32_t kr[4];
+                    ldmatrix_x4(kr, kaddr + ks * 32);
+                    mma_bf16_16816(s0, qa[ks][0], 0u, qa[ks][1], 0u, kr[0], kr[1]);
+                    mma_bf16_16816(s1, qa[ks][0], 0u, qa[ks][1], 0u, kr[2], kr[3]);
                 }
             }
+            // ---- scores of head g for the thread's four keys, in log2 units
+            float sc[4] = {s0[0], s0[1], s1[0], s1[1]};
+            const uint32_t fl[4] = {f01.x, f01.y, f23.x, f23.y};
+            float cm = -INFINITY;
 #pragma unroll
-            for (int gg = 0; gg < DEC_GMAX / 2 + 1; ++gg)
-#pragma unroll
-                for (int g = 0; g < DEC_GMAX; ++g)
-                    if (g == g_lo + gg) sc[g] = s2[gg].x + s2[gg].y;
-        }
-        // ---- per query head: chunk maximum, running maximum, probabilities, running sum
-#pragma unroll
-        for (int g = 0; g < DEC_GMAX; ++g) {
-            if (g >= g_lo && g < g_hi) {
-                float s = sc[g];
-                if (softcap > 0.f) s = tanhf(s * cap_in);
-                s = ((keep >> g) & 1u) ? s * sl2 : -INFINITY;
-                sc[g] = s;
-                float mx = s;
-#pragma unroll
-                for (int off = 16; off >= 1; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-                if (lane == 0) red[g * DEC_NW + warp] = mx;
+            for (int e = 0; e < 4; ++e) {
+                float x = sc[e];
+                if (softcap > 0.f) x = tanhf(x * cap_in);
+                x = ((fl[e] >> g) & 1u) ? x * sl2 : -INFINITY;
+                sc[e] = x;
+                cm = fmaxf(cm, x);
             }
-        }
-        __syncthreads();                        // maxima published; K tile no longer read
-        if (ch + 1 < c_end) copy_rows(kb, k_sn, kt, j0 + DEC_KEYS, keep_s[(ch + 1) & 1]);
-        else asm volatile("cp.async.commit_group;" ::: "memory");      // keep the group count uniform
-        float factor[DEC_GMAX], wsum[DEC_GMAX];
+            cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 1));
+            cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, 2));
+            const float m_new = fmaxf(m_run, cm);
+            const float factor = (m_run == -INFINITY) ? 0.f : exp2f(m_run - m_new);     // nothing accumulated yet: O and l are 0
+            float p[4], psum = 0.f;
 #pragma unroll
-        for (int g = 0; g < DEC_GMAX; ++g) {
-            factor[g] = 1.f; wsum[g] = 0.f;
-            if (g < G) {
-                float cm = red[g * DEC_NW];
+            for (int e = 0; e < 4; ++e) { p[e] = (m_new == -INFINITY) ? 0.f : exp2f(sc[e] - m_new); psum += p[e]; }
+            psum += __shfl_xor_sync(0xffffffffu, psum, 1);
+            psum += __shfl_xor_sync(0xffffffffu, psum, 2);
+            l_run = l_run * factor + psum;
+            m_run = m_new;
+            const uint32_t pa0 = dec_pack_bf16(p[0], p[1]), pa2 = dec_pack_bf16(p[2], p[3]);
+            // ---- O = O * factor + P V
+            {
+                const int mi = lane >> 3, mr = lane & 7;
+                const uint32_t vaddr = vst + (mr + 8 * (mi & 1)) * C::ROWB + 16 * (mi >> 1);
 #pragma unroll
-                for (int ww = 1; ww < DEC_NW; ++ww) cm = fmaxf(cm, red[g * DEC_NW + ww]);
-                const float m_new = fmaxf(m_run[g], cm);
-                factor[g] = (m_run[g] == -INFINITY) ? 0.f : exp2f(m_run[g] - m_new);    // nothing accumulated yet: O and l are 0
-                m_run[g] = m_new;
-                if (g >= g_lo && g < g_hi) {
-                    const float pj = (m_new == -INFINITY) ? 0.f : exp2f(sc[g] - m_new);   // -inf score -> 0
-                    ps[g * DEC_KEYS + key] = pj;
-                    float sum = pj;
-#pragma unroll
-                    for (int off = 16; off >= 1; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-                    wsum[g] = sum;
+                for (int np = 0; np < D / 16; ++np) {
+                    uint32_t vr[4];
+                    ldmatrix_x4_trans(vr, vaddr + np * 32);
+                    o[2 * np][0] *= factor; o[2 * np][1] *= factor;
+                    o[2 * np + 1][0] *= factor; o[2 * np + 1][1] *= factor;
+                    mma_bf16_16816(o[2 * np], pa0, 0u, pa2, 0u, vr[0], vr[1]);
+                    mma_bf16_16816(o[2 * np + 1], pa0, 0u, pa2, 0u, vr[2], vr[3]);
                 }
             }
         }
-        __syncthreads();                        // maxima consumed by everyone
-#pragma unroll
-        for (int g = 0; g < DEC_GMAX; ++g)
-            if (g >= g_lo && g < g_hi && lane == 0) red[g * DEC_NW + warp] = wsum[g];
-        asm volatile("cp.async.wait_group 1;" ::: "memory");   // V of this chunk has landed
-        __syncthreads();
-#pragma unroll
-        for (int g = 0; g < DEC_GMAX; ++g)
-            if (g < G) {
-                float ssum = red[g * DEC_NW];
-#pragma unroll
-                for (int ww = 1; ww < DEC_NW; ++ww) ssum += red[g * DEC_NW + ww];
-                l_run[g] = l_run[g] * factor[g] + ssum;
-            }
-        // ---- P V: 64 threads span the output dimensions, each group of 64 threads takes its share of the keys
-        {
-            const int quarter = t >> 6, dp = t & 63;
-#pragma unroll
-            for (int g = 0; g < DEC_GMAX; ++g)
-#pragma unroll
-                for (int e = 0; e < DPT; ++e) o_acc[g][e] *= factor[g];
-            for (int r = quarter * DEC_ROWS_PER_GROUP; r < (quarter + 1) * DEC_ROWS_PER_GROUP; r += 4) {
-                const uint4 kf = *reinterpret_cast<const uint4*>(&flags[r]);
-                if (!(kf.x | kf.y | kf.z | kf.w)) continue;              // uniform across the half: none of the four keys attended
-                float vv[4][DPT];
-#pragma unroll
-                for (int rr = 0; rr < 4; ++rr) {
-                    const unsigned char* vp = vt + (r + rr) * ROWB + dp * (2 * DPT);
-                    if constexpr (DPT == 1) {
-                        vv[rr][0] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(vp));
-                    } else if constexpr (DPT == 2) {
-                        const uint32_t u = *reinterpret_cast<const uint32_t*>(vp);
-                        vv[rr][0] = __uint_as_float(u << 16); vv[rr][1] = __uint_as_float(u & 0xffff0000u);
-                    } else {
-                        const uint2 u = *reinterpret_cast<const uint2*>(vp);
-                        vv[rr][0] = __uint_as_float(u.x << 16); vv[rr][1] = __uint_as_float(u.x & 0xffff0000u);
-                        vv[rr][2] = __uint_as_float(u.y << 16); vv[rr][3] = __uint_as_float(u.y & 0xffff0000u);
-                    }
-                }
-#pragma unroll
-                for (int g = 0; g < DEC_GMAX; ++g) {
-                    if (g < G) {
-                        const float4 p4 = *reinterpret_cast<const float4*>(ps + g * DEC_KEYS + r);
-#pragma unroll
-                        for (int e = 0; e < DPT; ++e) {
-                            float a = o_acc[g][e];
-                            a = fmaf(p4.x, vv[0][e], a); a = fmaf(p4.y, vv[1][e], a);
-                            a = fmaf(p4.z, vv[2][e], a); a = fmaf(p4.w, vv[3][e], a);
-                            o_acc[g][e] = a;
-                        }
-                    }
-                }
-            }
-        }
-        __syncthreads();                        // V tile, probabilities and flags of this chunk are free
-        keep = keep_next;
+        __syncwarp();                               // the stage may be refilled by the next issue
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    // ---- add the row groups, then the partial result of this split: [query head][split][2 + D] = (max, sum, O)
+    // ---- merge the warps of the CTA (through the ring, no longer needed), then one partial result per split:
+    //      [query head][split][2 + D] = (max, sum, O)
     __syncthreads();
-    float* xch = reinterpret_cast<float*>(kt);              // [row groups - 1][GMAX][D] (the K and V tiles are no longer needed)
-    const int quarter = t >> 6, dp = t & 63;
-    if (quarter > 0) {
+    float* xw = reinterpret_cast<float*>(smem_raw);             // [WARPS][GMAX][D + 2]
+    if (g < DEC_GMAX) {
+        float* dstw = xw + ((size_t)warp * DEC_GMAX + g) * (D + 2);
+        if (qd == 0) { dstw[0] = m_run; dstw[1] = l_run; }
 #pragma unroll
-        for (int g = 0; g < DEC_GMAX; ++g)
-#pragma unroll
-            for (int e = 0; e < DPT; ++e) xch[((quarter - 1) * DEC_GMAX + g) * D + dp * DPT + e] = o_acc[g][e];
+        for (int nt = 0; nt < D / 8; ++nt)
+            *reinterpret_cast<float2*>(dstw + 2 + nt * 8 + qd * 2) = make_float2(o[nt][0], o[nt][1]);
     }
     __syncthreads();
-    if (quarter == 0) {
+    for (int idx = threadIdx.x; idx < G * D; idx += C::WARPS * 32) {
+        const int gg = idx / D, d = idx % D;
+        float M = -INFINITY;
 #pragma unroll
-        for (int g = 0; g < DEC_GMAX; ++g) {
-            if (g < G) {
-                float* dst = part + (((size_t)b * Hq + hk * G + g) * nsplit + split) * (D + 2);
-                if (t == 0) { dst[0] = m_run[g]; dst[1] = l_run[g]; }
+        for (int ww = 0; ww < C::WARPS; ++ww) M = fmaxf(M, xw[((size_t)ww * DEC_GMAX + gg) * (D + 2)]);
+        float L = 0.f, acc = 0.f;
 #pragma unroll
-                for (int e = 0; e < DPT; ++e) {
-                    float a = o_acc[g][e];
-#pragma unroll
-                    for (int qq = 0; qq < DEC_ROWGROUPS - 1; ++qq) a += xch[(qq * DEC_GMAX + g) * D + dp * DPT + e];
-                    dst[2 + dp * DPT + e] = a;
-                }
-            }
+        for (int ww = 0; ww < C::WARPS; ++ww) {
+            const float* src = xw + ((size_t)ww * DEC_GMAX + gg) * (D + 2);
+            const float wgt = src[0] == -INFINITY ? 0.f : exp2f(src[0] - M);
+            L = fmaf(src[1], wgt, L);
+            acc = fmaf(src[2 + d], wgt, acc);
         }
+        float* dst = part + (((size_t)b * Hq + hk * G + gg) * nsplit + split) * (D + 2);
+        if (d == 0) { dst[0] = M; dst[1] = L; }
+        dst[2 + d] = acc;
     }
 }
 
-// one block per query head: merge the splits
+// one block per query head: merge the splits (weights of the splits once through shared memory, then every
+// thread one output dimension with independent loads)
 __global__ void __launch_bounds__(256)
 decode_merge_kernel(const float* __restrict__ part, int nsplit, int D, int Hq, __nv_bfloat16* __restrict__ o, int64_t o_sb,
                     int64_t o_sh, float* __restrict__ lse) {
-    const int hq = blockIdx.x;
+    __shared__ float wgt_s[512];
+    __shared__ float red_s[8];
+    const int hq = blockIdx.x, t = threadIdx.x;
     const float* p = part + (size_t)hq * nsplit * (D + 2);
-    float M = -INFINITY;
-    for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p[(size_t)s * (D + 2)]);
-    float L = 0.f;
-    for (int s = 0; s < nsplit; ++s) {
-        const float m = p[(size_t)s * (D + 2)];
-        if (m != -INFINITY) L += p[(size_t)s * (D + 2) + 1] * exp2f(m - M);
+    float m = -INFINITY;
+    for (int s = t; s < nsplit; s += 256) m = fmaxf(m, p[(size_t)s * (D + 2)]);
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    if ((t & 31) == 0) red_s[t >> 5] = m;
+    __syncthreads();
+    float M = red_s[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) M = fmaxf(M, red_s[i]);
+    __syncthreads();
+    float l = 0.f;
+    for (int s = t; s < nsplit; s += 256) {
+        const float ms = p[(size_t)s * (D + 2)];
+        const float wg = ms == -INFINITY ? 0.f : exp2f(ms - M);
+        wgt_s[s] = wg;
+        l = fmaf(p[(size_t)s * (D + 2) + 1], wg, l);
     }
-    for (int d = threadIdx.x; d < D; d += blockDim.x) {
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+    if ((t & 31) == 0) red_s[t >> 5] = l;
+    __syncthreads();
+    float L = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) L += red_s[i];
+    for (int d = t; d < D; d += 256) {
         float acc = 0.f;
-        for (int s = 0; s < nsplit; ++s) {
-            const float m = p[(size_t)s * (D + 2)];
-            if (m != -INFINITY) acc = fmaf(p[(size_t)s * (D + 2) + 2 + d], exp2f(m - M), acc);
-        }
+#pragma unroll 8
+        for (int s = 0; s < nsplit; ++s) acc = fmaf(p[(size_t)s * (D + 2) + 2 + d], wgt_s[s], acc);
         o[(size_t)(hq / Hq) * o_sb + (size_t)(hq % Hq) * o_sh + d] = __float2bfloat16(acc / L);
     }
-    if (threadIdx.x == 0) lse[hq] = (M + log2f(L)) * DEC_LN2;
+    if (t == 0) lse[hq] = (M + log2f(L)) * DEC_LN2;
 }
 
+static int decode_warps(int D) { return D == 256 ? 4 : 8; }
+
 static int decode_splits(const focus_shape* s) {
-    const int chunks = cdiv(s->n, DEC_KEYS);
+    const int groups = cdiv(s->n, DEC_GK);
     const int heads = s->batch * s->Hkv;
-    int want = cdiv(4 * 148, heads);                 // about four CTAs per SM in total (two rounds of two resident ones)
-    if (want > chunks) want = chunks;
+    int want = cdiv(2 * 148, heads);                 // about two CTAs per SM in total
+    const int max_useful = cdiv(groups, 4 * decode_warps(s->D));     // at least four steps per warp
+    if (want > max_useful) want = max_useful;
     if (want < 1) want = 1;
     if (want > 512) want = 512;
     return want;
@@ -329,19 +304,18 @@ template <int D>
 static int launch_decode_d(const focus_shape* s, const focus_tensor& q, const focus_tensor& k, const focus_tensor& v,
                            const uint32_t* mq_new, const uint32_t* mk, const focus_tensor& o, float* lse, float* part,
                            float scale, cudaStream_t st) {
+    using C = DecCfg<D>;
     const int nsplit = decode_splits(s);
-    const int chunks = cdiv(s->n, DEC_KEYS);
-    const int cps = cdiv(chunks, nsplit);
-    const size_t smem = (size_t)2 * DEC_KEYS * (2 * D + 16) + (size_t)DEC_GMAX * D * 4 + (size_t)DEC_GMAX * DEC_KEYS * 4 +
-                        (size_t)DEC_GMAX * DEC_NW * 4;
+    const int groups = cdiv(s->n, DEC_GK);
+    const int gps = cdiv(groups, nsplit);
     auto kern = decode_partial_kernel<D>;
-    int rc = check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
+    int rc = check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM),
                         "cudaFuncSetAttribute(decode)");
     if (rc) return rc;
-    kern<<<dim3(nsplit, s->batch * s->Hkv), DEC_THREADS, smem, st>>>(
+    kern<<<dim3(nsplit, s->batch * s->Hkv), C::WARPS * 32, C::SMEM, st>>>(
         reinterpret_cast<const __nv_bfloat16*>(q.ptr), q.stride_b, q.stride_h, reinterpret_cast<const __nv_bfloat16*>(k.ptr),
         k.stride_b, k.stride_h, k.stride_n, reinterpret_cast<const __nv_bfloat16*>(v.ptr), v.stride_b, v.stride_h, v.stride_n,
-        mq_new, mk, s->Hq, s->Hkv, s->Hq / s->Hkv, s->n, s->window, scale, s->softcap, nsplit, cps, part);
+        mq_new, mk, s->Hq, s->Hkv, s->Hq / s->Hkv, s->n, s->window, scale, s->softcap, nsplit, gps, part);
     if ((rc = check_cuda(cudaGetLastError(), "decode kernel launch"))) return rc;
     decode_merge_kernel<<<s->batch * s->Hq, 256, 0, st>>>(part, nsplit, D, s->Hq, reinterpret_cast<__nv_bfloat16*>(o.ptr),
                                                           o.stride_b, o.stride_h, lse);

@@ -1,6 +1,6 @@
 """focus_decode_step (one new query against the cached keys and values) vs the fp64 oracle's row n-1 of the
-forward definition.  fp32 arithmetic on bf16 values, probabilities not rounded: O max-abs <= 2e-2 (bf16 output
-rounding dominates), mean-abs <= 2e-3, lse max-abs <= 5e-3 -- the tolerances of the forward pass."""
+forward definition.  bf16 operands, fp32 accumulation, probabilities rounded to bf16 before P V: O max-abs <= 2e-2,
+mean-abs <= 2e-3, lse max-abs <= 5e-3 -- the tolerances of the forward pass."""
 import numpy as np
 import pytest
 import torch
