@@ -35,7 +35,7 @@ UNIT = "TFLOP/s"
 # DRAM bytes per launch of the attention kernel (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture per
 # entry, see profiles/), keyed by (workload name, layout); only valid for the kernel sources with this digest.
 ATTN_TRAFFIC = {("M-llama3-8b-128k", 1): 5.68e9}
-ATTN_TRAFFIC_SOURCES = "91fa7f96d5bbe61f"
+ATTN_TRAFFIC_SOURCES = "3b72e6b4b40c7aff"
 
 
 def attn_traffic(name, layout):

@@ -6,19 +6,28 @@
 //   warp 0        TMA producer: Q tiles once per item, then K and V tiles of every visited key tile
 //                 into a ring of shared-memory stages (128-byte swizzle)
 //   warp 1        MMA issuer: S_x = Q_x K^T and O_x += P_x V with tcgen05.mma, accumulators in TMEM
+//                 (the whole warp runs the loop, one elected lane issues)
 //   warps 4-7     softmax for query tile 0: tcgen05.ld S, mask, online max/sum, P (bf16) back to TMEM
 //   warps 8-11    softmax for query tile 1
-// The two softmax groups alternate on the tensor pipe: while one computes exponentials the MMAs of
-// the other run.  The running maximum is raised lazily (only when it grows by more than 2^8), and
-// then the owner of the row rescales its O row in TMEM itself.
+// After the split into roles the control warpgroup hands registers to the softmax warpgroups
+// (setmaxnreg).  The two softmax groups alternate on the tensor pipe: while one computes exponentials
+// the MMAs of the other run.  The running maximum is raised lazily (only when it grows by more than
+// 2^8), and then the owner of the row rescales its O row in TMEM itself.
 //
 // Head dimension 256 does not leave room in TMEM for two query tiles (O alone is 256 columns), so
 // there an item is a single 128-row query tile, S is double-buffered over consecutive key tiles
 // and one warpgroup does the softmax while the MMAs of the neighbouring tiles run.
 //
-// Which key tiles are visited: in dense mode every tile up to the diagonal; with a tiles
-// workspace, far tiles (every pair beyond the window) only when the live bitmap says the OR of the
-// query-tile masks meets the OR of the key-tile masks; near tiles always.
+// Which key tiles are visited, and in which order of items:
+//   dense mode      every tile up to the diagonal
+//   original layout far tiles (every pair beyond the window) only when the live bitmap says the OR
+//                   of the query-tile masks meets the OR of the key-tile masks; near tiles always
+//   class-sorted    Q, K, V are the copies gathered into the class-sorted order; per key class the
+//                   range of sorted key tiles listed for the query block; a row's kept columns of a
+//                   tile are a contiguous range found from the tile's ascending positions; O and lse
+//                   go straight to the rows' original positions
+// Items are laid out KV head by KV head (class-sorted: most key tiles first inside a group) and
+// dealt to the CTAs in alternating direction round by round.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 #include "tma_host.cuh"
