@@ -130,3 +130,27 @@ def test_cfg2_two_heads_all_rows_others_sampled():
     rows = [np.stack([np.full(wl.n, h), np.arange(wl.n)], 1) for h in (0, 31)]
     rows.append(fi.sample_rows(wl, 48))
     assert_parity(compare_rows(wl, Q, K, V, mq, mk, O, lse, rows=np.concatenate(rows)))
+
+
+@pytest.mark.parametrize("D", [64, 128, 256])
+@pytest.mark.parametrize("layout", [0, 1])
+def test_peaked_logits_exercise_the_lazy_rescale(D, layout):
+    """logit scale 8x the default: row maxima jump by far more than the rescale threshold between tiles, rows are
+    nearly one-hot, masked tiles precede the first attended key of many rows.  An output row is then close to a
+    single V row, values up to |4|, where the bf16 output grid alone is 2^-6 wide: the check is relative here,
+    |err| <= 2^-7 |O| + 1e-2 (P and O each rounded to bf16), with lse to the usual absolute tolerance."""
+    wl = fi.Workload("peak", 4, 2, D, 2300, 4, 1, 40, scale=8.0 / D ** 0.5, seed=90 + D)
+    Q, K, V, C = fi.make_inputs(wl, "cuda")
+    mq, mk = oracle_masks(wl, Q, K, C)
+    dq, dk = to_dev(mq), to_dev(mk)
+    ws, _ = gpu_tiles(wl, dq, dk, layout)
+    for dense in (False, True):
+        O, lse = gpu_attn(wl, Q, K, V) if dense else gpu_attn(wl, Q, K, V, dq, dk, ws, layout)
+        ref = fo.attn_rows(fi.bf16_bits(Q), fi.bf16_bits(K), fi.bf16_bits(V), mq, mk, wl.n + 1 if dense else wl.window,
+                           scale=wl.logit_scale)
+        og = O.float().cpu().numpy().reshape(-1, D).astype(np.float64)
+        assert np.isfinite(og).all()
+        err = np.abs(og - ref["O"])
+        assert (err <= 2.0 ** -7 * np.abs(ref["O"]) + 1e-2).all(), float(err.max())
+        assert err.mean() <= 2e-3
+        assert np.abs(lse.cpu().numpy().reshape(-1) - ref["lse"]).max() <= 5e-3
