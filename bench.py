@@ -211,6 +211,7 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=24576, help="oracle rows of the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the decode-step and router timings")
     ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
                     help="N > 1: weak = every rank runs the whole workload; strong = the KV heads of one workload are split over the ranks")
     ap.add_argument("--sweep", action="store_true", help="context-length sweep (one JSON line per point) instead of the bench line")
@@ -315,6 +316,55 @@ def main():
             dense_ms.append(a.elapsed_time(b))
     dense_ms = float(np.median(dense_ms))
 
+    # the two rows beyond the prefill path, timed alone (outside the timed steps): one decode step against the
+    # cached K/V of this workload (L2 flushed before every launch) and the paper's router on hidden states
+    extra = {}
+    if not args.no_extras:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+        def timed_alone(fn, reps=5):
+            ts = []
+            for i in range(reps + 1):
+                flush.zero_()
+                a, b = ev(), ev()
+                a.record(); fn(); b.record()
+                torch.cuda.synchronize()
+                if i > 0:
+                    ts.append(a.elapsed_time(b))
+            return float(np.median(ts))
+
+        if wl.G <= 8:
+            q_new, mq_new = Q[:, -1].contiguous(), mq[:, -1].contiguous()
+            o_dec = torch.empty((wl.Hq, wl.D), dtype=torch.bfloat16, device="cuda")
+            lse_dec = torch.empty(wl.Hq, dtype=torch.float32, device="cuda")
+            ws_dec = torch.empty(fb.focus_decode_workspace_bytes(shape), dtype=torch.uint8, device="cuda")
+            ms = timed_alone(lambda: fb.focus_decode_step(shape, q_new, K, V, mq_new, mk, o_dec, lse_dec, ws_dec))
+            # a K/V row pair is read when some query head of its KV head attends the key
+            union = torch.zeros(wl.Hkv, dtype=torch.int32, device="cuda")
+            for g in range(wl.G):
+                union |= mq_new.view(wl.Hkv, wl.G)[:, g]
+            far = wl.n - 1 - wl.window
+            rows = wl.Hkv * min(wl.n, wl.window + 1)
+            if far > 0:
+                rows += int(((mk[:, :far] & union[:, None]) != 0).sum().item())
+            gbs = (rows * 4 * wl.D + wl.Hkv * max(far, 0) * 4) / (ms * 1e-3) / 1e9
+            extra["focus_decode_step"] = dict(bound="hbm", ms=ms, achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s",
+                                              frac=gbs / peaks["hbm_gbs"], kv_rows_read=rows, kv_rows_total=wl.Hkv * wl.n,
+                                              note="bytes = 4 D per attended (KV head, key) + 4 per far key mask; L2 flushed")
+        d_model, d_g = 4096, 16
+        gen = torch.Generator(device="cuda"); gen.manual_seed(7)
+        hid = torch.randn((1, wl.n, d_model), generator=gen, device="cuda").to(torch.bfloat16)
+        Wg = torch.randn((d_model, d_g), generator=gen, device="cuda") / d_model ** 0.5
+        Cg = torch.randn((wl.K, d_g), generator=gen, device="cuda")
+        folded = torch.empty((wl.K, d_model), dtype=torch.float32, device="cuda")
+        mq_r, mk_r = torch.empty_like(mq), torch.empty_like(mk)
+        ms = timed_alone(lambda: fb.focus_assign_hidden(shape, hid, Wg, Cg, None, folded, mq_r, mk_r))
+        gbs = (wl.n * d_model * 2 + (wl.Hq + wl.Hkv) * wl.n * 4) / (ms * 1e-3) / 1e9
+        extra["focus_assign_hidden"] = dict(bound="hbm", ms=ms, achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s",
+                                            frac=gbs / peaks["hbm_gbs"],
+                                            note=f"hidden states [n, {d_model}] bf16, d_g = {d_g}; bytes = 2 d_model per token + the mask rows written")
+        del hid, flush
+
     # whole-job work: replicas of the workload (weak) or the one workload split by heads (strong)
     job_flop = world * kept_flop if args.scaling == "weak" else multi.sum_over_ranks(kept_flop, dist, "cuda")
     value = job_flop / (ms_step * 1e-3) / 1e12
@@ -389,7 +439,8 @@ def main():
                                   peak=peaks["hbm_gbs"], unit="GB/s",
                                   frac=(wl.Hq + wl.Hkv) * wl.n * (2 * wl.D + 4) / (t_assign * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                   note="two launches (Q heads, K heads); bytes = (2 D + 4) per head vector"),
-                focus_build_tiles=dict(ms=t_tiles, note="integer passes over the masks; launch-latency bound at this size")),
+                focus_build_tiles=dict(ms=t_tiles, note="integer passes over the masks; launch-latency bound at this size"),
+                **extra),
             breakdown=dict(assign_ms=t_assign, build_tiles_ms=t_tiles, attn_ms=t_attn, dense_attn_ms=dense_ms,
                            speedup_vs_dense=dense_ms / t_attn, dense_tflops=dense_flop / (dense_ms * 1e-3) / 1e12,
                            kept_pairs=kept, kept_fraction=kept / wl.dense_pairs(), far_tiles=counters[0],
