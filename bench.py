@@ -256,8 +256,8 @@ def main():
     O = torch.empty_like(Q)
     lse = torch.empty((wl.Hq, wl.n), dtype=torch.float32, device="cuda")
     status = torch.zeros(4, dtype=torch.int32, device="cuda")
-    # assign x2, build_tiles (3 kernels; class-sorted: + 6 per side + ranges + order), attention (+ 3 gathers)
-    launches_per_step = 2 + 3 + 1 + (14 + 3 if layout == 1 else 0)
+    # assign x2, build_tiles (4 kernels; class-sorted: + 6 per side + ranges + order), attention (+ 3 gathers)
+    launches_per_step = 2 + 4 + 1 + (14 + 3 if layout == 1 else 0)
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
     marks = []

@@ -91,6 +91,7 @@ typedef struct {
     size_t gbits;      /* uint32 [B*Hkv][nkt][K][4]: bit j of word j/32 set when key 128*b + j is in group g */
     size_t live;       /* uint32 [B*Hq][nqt][nkw]: bit b set when (a, b) is a far tile pair that may hold a kept pair */
     size_t live_cnt;   /* int32  [B*Hq][nqt]: popcount of the row of `live` */
+    size_t kany, kall; /* uint32 [B*Hkv][K][nkw]: bit b set when key tile b holds a member of group g / only members of g */
     /* class-sorted layout only (0 otherwise) */
     int32_t nqp, nkp;  /* capacity of the sorted arrays in rows (multiples of 256): n + room for padding every class segment */
     size_t ncls_q, ncls_k;   /* int32 [B*Hq], [B*Hkv]: distinct mask values of the head */

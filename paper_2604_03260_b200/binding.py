@@ -32,6 +32,7 @@ class focus_tiles_layout(C.Structure):
                 ("total_bytes", C.c_size_t), ("counters", C.c_size_t),
                 ("orq", C.c_size_t), ("andq", C.c_size_t), ("ork", C.c_size_t), ("andk", C.c_size_t),
                 ("gbits", C.c_size_t), ("live", C.c_size_t), ("live_cnt", C.c_size_t),
+                ("kany", C.c_size_t), ("kall", C.c_size_t),
                 ("nqp", C.c_int32), ("nkp", C.c_int32),
                 ("ncls_q", C.c_size_t), ("ncls_k", C.c_size_t), ("cls_q", C.c_size_t), ("cls_k", C.c_size_t),
                 ("cnt_q", C.c_size_t), ("cnt_k", C.c_size_t),

@@ -89,6 +89,8 @@ static int layout_of(const focus_shape* s, int layout, focus_tiles_layout* L) {
     L->gbits = take(HK * L->nkt * (size_t)s->K * 4 * 4);
     L->live = take(HQ * L->nqt * (size_t)L->nkw * 4);
     L->live_cnt = take(HQ * L->nqt * 4);
+    L->kany = take(HK * (size_t)s->K * L->nkw * 4);
+    L->kall = take(HK * (size_t)s->K * L->nkw * 4);
     if (layout == FOCUS_LAYOUT_CLASS_SORTED) {
         L->nqp = sorted_capacity(s->n);
         L->nkp = sorted_capacity(s->n);

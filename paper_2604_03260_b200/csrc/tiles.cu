@@ -40,51 +40,79 @@ summarise_kernel(const uint32_t* __restrict__ m, int n, int nt, int K, uint32_t*
     }
 }
 
-// far(a, b): every pair of query tile a and key tile b has i - j > w
-__device__ __forceinline__ bool tile_pair_far(int a, int b, int n, int w) {
-    const long long qmin = (long long)a * TM;
-    const long long kmax = min((long long)n, (long long)(b + 1) * TN) - 1;
-    return qmin - kmax > (long long)w;
+// Per KV head and group g: which key tiles hold a member of g (from the OR summaries) and which key tiles
+// consist of members of g only (from the AND summaries), as bitmaps over the key tiles.  thread = (head, word).
+__global__ void __launch_bounds__(256)
+group_tiles_kernel(const uint32_t* __restrict__ ork, const uint32_t* __restrict__ andk, int HK, int nkt, int nkw, int K,
+                   uint32_t* __restrict__ kany, uint32_t* __restrict__ kall) {
+    const int gid = blockIdx.x * blockDim.x + threadIdx.x;
+    if (gid >= HK * nkw) return;
+    const int hk = gid / nkw, wd = gid % nkw;
+    uint32_t any_w[32], all_w[32];
+#pragma unroll
+    for (int g = 0; g < 32; ++g) any_w[g] = all_w[g] = 0u;
+    for (int c = 0; c < 32; ++c) {
+        const int b = wd * 32 + c;
+        if (b >= nkt) break;
+        const uint32_t o = ork[(size_t)hk * nkt + b], a = andk[(size_t)hk * nkt + b];
+#pragma unroll
+        for (int g = 0; g < 32; ++g) {
+            any_w[g] |= ((o >> g) & 1u) << c;
+            all_w[g] |= ((a >> g) & 1u) << c;
+        }
+    }
+    for (int g = 0; g < K; ++g) {
+        kany[((size_t)hk * K + g) * nkw + wd] = any_w[g];
+        kall[((size_t)hk * K + g) * nkw + wd] = all_w[g];
+    }
 }
 
-// One block per (query tile, head); threads stride over the bitmap words of the row.
+// Live far-tile bitmap.  Key tile b is far for query tile a when every pair has i - j > w, i.e. b < (128 a - w) / 128;
+// a far tile is live when the query tile's OR summary meets the key tile's, full when the AND summaries meet.  A word
+// of the bitmap is the OR, over the groups present in the query tile, of the groups' key-tile bitmaps.
+// One block per (query tile, head); threads stride over the words of the row.
 __global__ void __launch_bounds__(128)
-live_kernel(const uint32_t* __restrict__ orq, const uint32_t* __restrict__ andq, const uint32_t* __restrict__ ork,
-            const uint32_t* __restrict__ andk, int G_heads, int Hq, int Hkv, int n, int w, int nqt, int nkt, int nkw,
+live_kernel(const uint32_t* __restrict__ orq, const uint32_t* __restrict__ andq, const uint32_t* __restrict__ kany,
+            const uint32_t* __restrict__ kall, int G_heads, int Hq, int Hkv, int w, int K, int nqt, int nkw,
             uint32_t* __restrict__ live, int32_t* __restrict__ live_cnt, unsigned long long* counters) {
     const int a = blockIdx.x, hq = blockIdx.y;
     const int b_idx = hq / Hq, h = hq % Hq;
     const int hk = b_idx * Hkv + h / G_heads;
     const uint32_t oq = orq[(size_t)hq * nqt + a], aq = andq[(size_t)hq * nqt + a];
-    unsigned int nfar = 0, nlive = 0, nfull = 0;
+    const long long d = (long long)a * TM - w;
+    const int nfar_tiles = d > 0 ? (int)(d / TN) : 0;                 // far tiles are the first nfar_tiles key tiles
+    unsigned int nlive = 0, nfull = 0;
     for (int wd = threadIdx.x; wd < nkw; wd += blockDim.x) {
-        uint32_t bits = 0;
-        for (int c = 0; c < 32; ++c) {
-            const int b = wd * 32 + c;
-            if (b >= nkt) break;
-            if (!tile_pair_far(a, b, n, w)) break;      // far tiles are a prefix of the row
-            ++nfar;
-            const uint32_t ok = ork[(size_t)hk * nkt + b];
-            if (oq & ok) {
-                bits |= 1u << c;
-                ++nlive;
-                if (aq & andk[(size_t)hk * nkt + b]) ++nfull;
+        const int rem = nfar_tiles - wd * 32;
+        const uint32_t far_mask = rem >= 32 ? 0xffffffffu : (rem <= 0 ? 0u : ((1u << rem) - 1u));
+        uint32_t lv = 0, fl = 0;
+        if (far_mask) {
+            for (uint32_t m = oq; m; m &= m - 1) {
+                const int g = __ffs(m) - 1;
+                if (g < K) lv |= kany[((size_t)hk * K + g) * nkw + wd];
             }
+            for (uint32_t m = aq; m; m &= m - 1) {
+                const int g = __ffs(m) - 1;
+                if (g < K) fl |= kall[((size_t)hk * K + g) * nkw + wd];
+            }
+            lv &= far_mask;
+            fl &= far_mask;
         }
-        live[((size_t)hq * nqt + a) * nkw + wd] = bits;
+        live[((size_t)hq * nqt + a) * nkw + wd] = lv;
+        nlive += __popc(lv);
+        nfull += __popc(fl);
     }
-    __shared__ unsigned int s[3];
-    if (threadIdx.x < 3) s[threadIdx.x] = 0;
+    __shared__ unsigned int s[2];
+    if (threadIdx.x < 2) s[threadIdx.x] = 0;
     __syncthreads();
-    if (nfar) atomicAdd(&s[0], nfar);
-    if (nlive) atomicAdd(&s[1], nlive);
-    if (nfull) atomicAdd(&s[2], nfull);
+    if (nlive) atomicAdd(&s[0], nlive);
+    if (nfull) atomicAdd(&s[1], nfull);
     __syncthreads();
     if (threadIdx.x == 0) {
-        live_cnt[(size_t)hq * nqt + a] = (int32_t)s[1];
-        if (s[0]) atomicAdd(&counters[0], (unsigned long long)s[0]);
-        if (s[1]) atomicAdd(&counters[1], (unsigned long long)s[1]);
-        if (s[2]) atomicAdd(&counters[2], (unsigned long long)s[2]);
+        live_cnt[(size_t)hq * nqt + a] = (int32_t)s[0];
+        if (nfar_tiles) atomicAdd(&counters[0], (unsigned long long)nfar_tiles);
+        if (s[0]) atomicAdd(&counters[1], (unsigned long long)s[0]);
+        if (s[1]) atomicAdd(&counters[2], (unsigned long long)s[1]);
     }
 }
 
@@ -149,8 +177,11 @@ int launch_build_tiles(const focus_shape* s, const uint32_t* mq, const uint32_t*
     auto* gb = reinterpret_cast<uint32_t*>(ws + L.gbits);
     summarise_kernel<<<dim3(L.nqt, HQ), 128, 0, st>>>(mq, s->n, L.nqt, s->K, orq, andq, nullptr);
     summarise_kernel<<<dim3(L.nkt, HK), 128, 0, st>>>(mk, s->n, L.nkt, s->K, ork, andk, gb);
-    live_kernel<<<dim3(L.nqt, HQ), 128, 0, st>>>(orq, andq, ork, andk, s->Hq / s->Hkv, s->Hq, s->Hkv, s->n, s->window,
-                                                 L.nqt, L.nkt, L.nkw, reinterpret_cast<uint32_t*>(ws + L.live),
+    auto* kany = reinterpret_cast<uint32_t*>(ws + L.kany);
+    auto* kall = reinterpret_cast<uint32_t*>(ws + L.kall);
+    group_tiles_kernel<<<cdiv(HK * L.nkw, 256), 256, 0, st>>>(ork, andk, HK, L.nkt, L.nkw, s->K, kany, kall);
+    live_kernel<<<dim3(L.nqt, HQ), 128, 0, st>>>(orq, andq, kany, kall, s->Hq / s->Hkv, s->Hq, s->Hkv, s->window, s->K, L.nqt,
+                                                 L.nkw, reinterpret_cast<uint32_t*>(ws + L.live),
                                                  reinterpret_cast<int32_t*>(ws + L.live_cnt),
                                                  reinterpret_cast<unsigned long long*>(ws + L.counters));
     if ((rc = check_cuda(cudaGetLastError(), "build_tiles kernels"))) return rc;
