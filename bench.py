@@ -379,11 +379,34 @@ def main():
         h2d = sum(x.numel() * x.element_size() for x in (hQ, hK, hV, hC))
         d2h = sum(x.numel() * x.element_size() for x in (hO, hL))
 
+        # The path shards by KV head with no exchange step, so the host-buffer pass is pipelined over the KV-head
+        # groups on two streams: copies of one group (in and out) overlap the kernels of its neighbour.
+        G = wl.G
+        shape_g = fb.make_shape(G, 1, wl.n, wl.D, wl.K, wl.topk, wl.window, wl.scale, wl.softcap)
+        streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        ws_g = [fb.alloc_workspace(shape_g, layout) for _ in streams]
+
         def e2e_step():
-            Q.copy_(hQ, non_blocking=True); K.copy_(hK, non_blocking=True)
-            V.copy_(hV, non_blocking=True); C.copy_(hC, non_blocking=True)
-            step(False)
-            hO.copy_(O, non_blocking=True); hL.copy_(lse, non_blocking=True)
+            start = ev()
+            start.record()
+            for st in streams:
+                st.wait_event(start)
+            for g in range(wl.Hkv):
+                st = streams[g % 2]
+                qs_, ks_ = slice(g * G, (g + 1) * G), slice(g, g + 1)
+                with torch.cuda.stream(st):
+                    Q[qs_].copy_(hQ[qs_], non_blocking=True); K[ks_].copy_(hK[ks_], non_blocking=True)
+                    V[ks_].copy_(hV[ks_], non_blocking=True); C[ks_].copy_(hC[ks_], non_blocking=True)
+                    fb.focus_assign(shape_g, Q[qs_], G, C[ks_], mq[qs_], near, stream=st)
+                    fb.focus_assign(shape_g, K[ks_], 1, C[ks_], mk[ks_], near, stream=st)
+                    fb.focus_build_tiles(shape_g, mq[qs_], mk[ks_], layout, ws_g[g % 2], stream=st)
+                    fb.focus_attn_fwd(shape_g, Q[qs_], K[ks_], V[ks_], mq[qs_], mk[ks_], ws_g[g % 2], layout, O[qs_], lse[qs_],
+                                      status, stream=st)
+                    hO[qs_].copy_(O[qs_], non_blocking=True); hL[qs_].copy_(lse[qs_], non_blocking=True)
+            for st in streams:
+                done = ev()
+                done.record(st)
+                torch.cuda.current_stream().wait_event(done)
 
         e2e_step()
         barrier()
@@ -395,10 +418,16 @@ def main():
         b.record()
         barrier()
         e2e_ms = a.elapsed_time(b) / nrep
+        # what came back over the bus is what the one-launch path computes (heads are independent: bit for bit)
+        step(False)
+        torch.cuda.synchronize()
+        assert torch.equal(hO, O.cpu()) and torch.equal(hL, lse.cpu()), "pipelined host-buffer pass differs from the device pass"
         e2e_ms = multi.max_over_ranks(e2e_ms, dist, "cuda")
         e2e = dict(value=job_flop / (e2e_ms * 1e-3) / 1e12, unit=UNIT, h2d_bytes_per_step=int(h2d),
-                   d2h_bytes_per_step=int(d2h), ms_per_step=e2e_ms)
-        del hQ, hK, hV, hO, hL
+                   d2h_bytes_per_step=int(d2h), ms_per_step=e2e_ms,
+                   how="pinned host buffers; per KV-head group: H2D of its Q/K/V/centroids, assign, build_tiles, attention, "
+                       "D2H of its O/lse; groups alternate on two streams")
+        del hQ, hK, hV, hO, hL, ws_g
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
