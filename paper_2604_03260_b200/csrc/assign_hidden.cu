@@ -10,7 +10,7 @@
 
 namespace focus {
 
-constexpr int AH_THREADS = 128;      // tokens per block
+constexpr int AH_THREADS = 64;       // tokens per block (small, so that modest sequence lengths still fill the GPU)
 constexpr int AH_CHUNK = 64;         // elements of a row per stage
 constexpr int AH_ROWB = 2 * AH_CHUNK + 16;   // padded row: conflict-free 16-byte reads per token
 
