@@ -206,7 +206,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="focus", choices=["focus", "reference"])
     ap.add_argument("--workload", default="M128k")
-    ap.add_argument("--layout", type=int, default=1, help="0 = original token order, 1 = class-sorted (group-permuted)")
+    ap.add_argument("--layout", type=int, default=1, help="0 = original token order, 1 = class-sorted (group-permuted), 2 = chosen by the library from the shape")
     ap.add_argument("--ref-rows", type=int, default=2048, help="oracle rows per step (reference arm)")
     ap.add_argument("--cpu-rows", type=int, default=24576, help="oracle rows of the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -237,7 +237,6 @@ def main():
         multi.barrier(dist)
 
     peaks = load_peaks()
-    layout = args.layout
     Q, K, V, C = fi.make_inputs(wl, "cuda")
     wl_full = wl
     if args.scaling == "strong" and world > 1:
@@ -249,6 +248,7 @@ def main():
         Q, K, V, C = Q[q0:q1].contiguous(), K[k0:k1].contiguous(), V[k0:k1].contiguous(), C[k0:k1].contiguous()
         wl = replace(wl, Hq=q1 - q0, Hkv=k1 - k0)
     shape = fb.shape_of(wl)
+    layout = fb.focus_tiles_layout_of(shape, args.layout).layout         # 2 = chosen by the library, resolved here
     mq = torch.empty((wl.Hq, wl.n), dtype=torch.int32, device="cuda")
     mk = torch.empty((wl.Hkv, wl.n), dtype=torch.int32, device="cuda")
     near = torch.zeros(1, dtype=torch.int64, device="cuda")

@@ -74,6 +74,12 @@ typedef struct {
 
 #define FOCUS_LAYOUT_ORIGINAL 0
 #define FOCUS_LAYOUT_CLASS_SORTED 1
+/* Let the library choose between the two from the shape alone (n, K, topk): the class-sorted layout when the
+ * sequence is long enough for its fixed costs (at least 16384 tokens and 2048 per mask class, C(K, topk) classes
+ * assumed) and enough distant pairs fall away (at least half of them for uniform memberships, or at least 15 % from
+ * 65536 tokens on); the original layout otherwise.  focus_tiles_layout_of reports the choice in `layout`; pass
+ * the same value to focus_tiles_workspace_bytes, focus_build_tiles and focus_attn_fwd. */
+#define FOCUS_LAYOUT_AUTO 2
 
 /*
  * Byte offsets of the arrays inside a tiles workspace (a pure function of shape and layout;

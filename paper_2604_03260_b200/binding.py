@@ -14,6 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libfocus_b200.so")
 
 FOCUS_LAYOUT_ORIGINAL = 0
 FOCUS_LAYOUT_CLASS_SORTED = 1
+FOCUS_LAYOUT_AUTO = 2
 FOCUS_MAX_CLASSES = 64
 
 

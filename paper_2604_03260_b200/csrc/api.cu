@@ -67,12 +67,32 @@ int require_sm100() {
     return FOCUS_OK;
 }
 
+// C(a, b) as a double (a <= 32)
+static double binom(int a, int b) {
+    if (b < 0 || b > a) return 0.0;
+    double r = 1.0;
+    for (int j = 0; j < b; ++j) r = r * (a - j) / (j + 1);
+    return r;
+}
+
+// FOCUS_LAYOUT_AUTO: a function of the shape alone, so that every entry point resolves it alike
+static int choose_layout(const focus_shape* s) {
+    const double classes = binom(s->K, s->topk);
+    if (classes > (double)FOCUS_MAX_CLASSES + 0.5) return FOCUS_LAYOUT_ORIGINAL;
+    const double dropped = binom(s->K - s->topk, s->topk) / classes;      // far pairs without a shared group, uniform memberships
+    const double min_n = classes * 2048.0 > 16384.0 ? classes * 2048.0 : 16384.0;
+    if ((double)s->n < min_n) return FOCUS_LAYOUT_ORIGINAL;
+    if (dropped >= 0.5 || (s->n >= 65536 && dropped >= 0.15)) return FOCUS_LAYOUT_CLASS_SORTED;
+    return FOCUS_LAYOUT_ORIGINAL;
+}
+
 static int layout_of(const focus_shape* s, int layout, focus_tiles_layout* L) {
     int rc = validate_shape(s);
     if (rc) return rc;
     if (!L) return fail(FOCUS_ERR_INVALID_ARG, "out is NULL");
+    if (layout == FOCUS_LAYOUT_AUTO) layout = choose_layout(s);
     if (layout != FOCUS_LAYOUT_ORIGINAL && layout != FOCUS_LAYOUT_CLASS_SORTED)
-        return fail(FOCUS_ERR_INVALID_ARG, "layout must be 0 (original) or 1 (class-sorted)");
+        return fail(FOCUS_ERR_INVALID_ARG, "layout must be 0 (original), 1 (class-sorted) or 2 (chosen by the library)");
     memset(L, 0, sizeof *L);
     const size_t HQ = (size_t)s->batch * s->Hq, HK = (size_t)s->batch * s->Hkv;
     L->layout = layout;
@@ -184,6 +204,7 @@ int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, const uint32
     if ((uintptr_t)ws % 256) return fail(FOCUS_ERR_INVALID_ARG, "ws is not 256-byte aligned");
     if (ws_bytes < L.total_bytes)
         return fail(FOCUS_ERR_CAPACITY, "workspace has %zu bytes, %zu needed", ws_bytes, L.total_bytes);
+    layout = L.layout;                     // FOCUS_LAYOUT_AUTO resolved
     if (layout == FOCUS_LAYOUT_CLASS_SORTED) {
         // masks with exactly topk bits have C(K, topk) values; more than the class table holds is refused here,
         // other mask patterns with too many values are caught on the device (counters[4], then dev_status)

@@ -97,3 +97,16 @@ def test_without_a_device_the_library_reports_an_error_instead_of_computing():
     t_ok = fb.focus_tensor(4096, 8 * 1000 * 128, 1000 * 128, 128)
     rc = fb.lib().focus_assign(ctypes.byref(s), t_ok, 8, 4096, 4096, None, 1e-5, None)
     assert rc in (-4, -5)
+
+
+def test_auto_layout_is_resolved_from_the_shape():
+    pick = lambda Hq, Hkv, n, K, t: fb.focus_tiles_layout_of(fb.make_shape(Hq, Hkv, n, 128, K, t, 2048), fb.FOCUS_LAYOUT_AUTO).layout
+    assert pick(32, 8, 8192, 4, 1) == 0 and pick(32, 8, 16384, 4, 1) == 1          # top-1 of 4: 3/4 of far pairs fall away
+    assert pick(32, 8, 32768, 4, 2) == 0 and pick(32, 8, 131072, 4, 2) == 1        # top-2 of 4: only 1/6 fall away
+    assert pick(32, 8, 16384, 8, 1) == 1
+    assert pick(32, 8, 32768, 8, 2) == 0 and pick(32, 8, 65536, 8, 2) == 1         # 28 classes need 2048 tokens each
+    assert pick(4, 2, 1 << 20, 32, 3) == 0                                          # more classes than the sorted layout holds
+    s = fb.make_shape(32, 8, 131072, 128, 4, 2, 2048)
+    assert fb.focus_tiles_workspace_bytes(s, fb.FOCUS_LAYOUT_AUTO) == fb.focus_tiles_workspace_bytes(s, 1)
+    L = fb.focus_tiles_layout()
+    assert fb.lib().focus_tiles_layout_of(ctypes.byref(s), 3, ctypes.byref(L)) == -1

@@ -158,3 +158,10 @@ def test_cfg2_sorted_two_heads_all_rows_others_sampled():
     rows = [np.stack([np.full(wl.n, h), np.arange(wl.n)], 1) for h in (3, 28)]
     rows.append(fi.sample_rows(wl, 48))
     assert_parity(compare_rows(wl, Q, K, V, mq, mk, O, lse, rows=np.concatenate(rows)))
+
+
+def test_auto_layout_runs_whichever_it_picks():
+    for wl, expect in ((fi.Workload("a0", 4, 2, 128, 3000, 4, 1, 64, seed=51), 0),
+                       (fi.Workload("a1", 4, 2, 128, 17000, 4, 1, 64, seed=52), 1)):
+        assert fb.focus_tiles_layout_of(fb.shape_of(wl), fb.FOCUS_LAYOUT_AUTO).layout == expect
+        run_case(wl, layout=fb.FOCUS_LAYOUT_AUTO, rows=fi.sample_rows(wl, 200))
