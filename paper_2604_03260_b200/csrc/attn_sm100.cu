@@ -46,7 +46,7 @@ constexpr int EX2_POLY_PER_8 = 0;
 // gives most of its share to the softmax warpgroups.
 constexpr int REGS_CONTROL = 96;
 constexpr int REGS_SOFTMAX_2WG = 200;        // 128*96 + 256*200 = 63488 <= 65536
-constexpr int REGS_SOFTMAX_1WG = 232;        // 128*96 + 128*232
+constexpr int REGS_SOFTMAX_1WG = 232;        // 128*96 + 128*232 (unused while a single query tile is split over two warpgroups)
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
@@ -181,16 +181,25 @@ struct AttnCfg {
     static constexpr int SUBT = D / 64;
     static constexpr uint32_t SUB_BYTES = 128 * 64 * 2;
     static constexpr uint32_t TILE_BYTES = SUB_BYTES * SUBT;
+    // The K/V ring: a stage holds a whole 128-key tile of K or of V.  At D = 256 only two stages fit next to Q.
     static constexpr int NSTAGE = (D == 256) ? 2 : ((D == 128) ? 5 : 8);
     static constexpr uint32_t SMEM_BYTES = 1024 + NQ * TILE_BYTES + NSTAGE * TILE_BYTES;
+    // Ring order of the tiles.  With one query tile the S of the next key tile is issued before the current P V, so
+    // K(next) travels ahead of V(current); with two query tiles V(current) is consumed and released first.
+    static constexpr bool K_AHEAD = NQ == 1;
     static constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O0 = 256, COL_O1 = 256 + D;
-    static constexpr int THREADS = 128 + 128 * NQ;
+    // With a single query tile two threads share a row: each of the two softmax warpgroups owns one 64-column
+    // half of every key tile (its S columns, its P columns, its part of the row sum) and one half of the O row.
+    static constexpr int NSPLIT = NQ == 1 ? 2 : 1;
+    static constexpr int NC = 128 / NSPLIT;                  // S columns per softmax thread
+    static constexpr int THREADS = 128 + 128 * NQ * NSPLIT;
 };
 
 struct SharedCtl {
     uint64_t q_full, q_empty;
     uint64_t s_full[2], p_full[2], o_full[2];
     uint64_t pv_done;
+    uint64_t xchg[4];                 // split rows, per 32-row quadrant: both column halves have published a per-row value
     uint64_t kv_full[8], kv_empty[8];
     uint32_t tmem_base;
     int abort_flag;
@@ -344,6 +353,9 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     constexpr int NQ = C::NQ;
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) SharedCtl ctl;
+    // split rows: [parity][column half][row] row maxima, at the end row sums (the other instantiations have no room to spare)
+    __shared__ float xval_s[C::NSPLIT == 2 ? 2 * 2 * 128 : 1];
+    auto xval = [&](int par, int hf, int row) -> float& { return xval_s[C::NSPLIT == 2 ? (par * 2 + hf) * 128 + row : 0]; };
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sq = base;                                 // NQ query tiles
     const uint32_t skv = base + NQ * C::TILE_BYTES;            // ring of K / V tiles
@@ -359,9 +371,10 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         mbar_init(smem_u32(&ctl.q_full), 1);
         mbar_init(smem_u32(&ctl.q_empty), 1);
         mbar_init(smem_u32(&ctl.pv_done), 1);
+        for (int qd = 0; qd < 4; ++qd) mbar_init(smem_u32(&ctl.xchg[qd]), 2);
         for (int x = 0; x < 2; ++x) {
             mbar_init(smem_u32(&ctl.s_full[x]), 1);
-            mbar_init(smem_u32(&ctl.p_full[x]), 128);
+            mbar_init(smem_u32(&ctl.p_full[x]), 128 * C::NSPLIT);
             mbar_init(smem_u32(&ctl.o_full[x]), 1);
         }
         for (int s = 0; s < C::NSTAGE; ++s) {
@@ -405,21 +418,37 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     for (int c = 0; c < C::SUBT; ++c)
                         tma_load_4d(sq + x * C::TILE_BYTES + c * C::SUB_BYTES, &tm_q, smem_u32(&ctl.q_full), c * 64,
                                     (A * NQ + x) * 128, qh, qb);
-                for (; ok && kb >= 0; kb = walk.next()) {
-                    for (int kv = 0; kv < 2; ++kv) {
-                        const int slot = (int)(nload % C::NSTAGE);
-                        const long long use = nload / C::NSTAGE;
-                        if (use > 0 && !ctl_wait(&ctl.kv_empty[slot], (uint32_t)((use - 1) & 1), &ctl)) {
-                            report_timeout(p, &ctl, 11, (int)item);
-                            ok = false;
-                            break;
-                        }
-                        const uint32_t bar = smem_u32(&ctl.kv_full[slot]);
-                        mbar_arrive_expect_tx(bar, C::TILE_BYTES);
-                        for (int c = 0; c < C::SUBT; ++c)
-                            tma_load_4d(skv + slot * C::TILE_BYTES + c * C::SUB_BYTES, kv ? &tm_v : &tm_k, bar, c * 64,
-                                        kb * 128, kh, qb);
-                        ++nload;
+                // one K or V tile into the next stage of the ring
+                auto load_tile = [&](bool is_v, int tile) {
+                    const int slot = (int)(nload % C::NSTAGE);
+                    const long long use = nload / C::NSTAGE;
+                    if (use > 0 && !ctl_wait(&ctl.kv_empty[slot], (uint32_t)((use - 1) & 1), &ctl)) {
+                        report_timeout(p, &ctl, 11, (int)item);
+                        ok = false;
+                        return;
+                    }
+                    const uint32_t bar = smem_u32(&ctl.kv_full[slot]);
+                    mbar_arrive_expect_tx(bar, C::TILE_BYTES);
+                    for (int c = 0; c < C::SUBT; ++c)
+                        tma_load_4d(skv + slot * C::TILE_BYTES + c * C::SUB_BYTES, is_v ? &tm_v : &tm_k, bar, c * 64, tile * 128,
+                                    kh, qb);
+                    ++nload;
+                };
+                if constexpr (C::K_AHEAD) {
+                    // load order K(0), then per tile K(next), V(current): the K of the next tile is needed first (its
+                    // S is issued before the current P V) and so travels ahead of the V it shares the ring with
+                    load_tile(false, kb);
+                    while (ok && kb >= 0) {
+                        const int nxt = walk.next();
+                        if (nxt >= 0) load_tile(false, nxt);
+                        if (ok) load_tile(true, kb);
+                        kb = nxt;
+                    }
+                } else {
+                    // two query tiles: V(current) is consumed and released before K(next), so it goes first
+                    for (; ok && kb >= 0; kb = walk.next()) {
+                        load_tile(false, kb);
+                        if (ok) load_tile(true, kb);
                     }
                 }
                 ++it;
@@ -446,11 +475,10 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (elect_one()) {
                     const uint32_t d = tmem + (buf ? C::COL_S1 : C::COL_S0);
                     const uint64_t ad = qdesc0 + (uint64_t)((x * C::TILE_BYTES) >> 4);
-                    const uint64_t bd = kvdesc0 + (uint64_t)((kslot * C::TILE_BYTES) >> 4);
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks) {
                         const uint64_t off = (uint64_t)(((ks / 4) * C::SUB_BYTES + (ks % 4) * 32) >> 4);
-                        umma_ss(d, ad + off, bd + off, IDESC_S, ks > 0);
+                        umma_ss(d, ad + off, kvdesc0 + (uint64_t)((kslot * C::TILE_BYTES) >> 4) + off, IDESC_S, ks > 0);
                     }
                 }
             };
@@ -460,14 +488,19 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     const uint32_t d = tmem + (x ? C::COL_O1 : C::COL_O0);
                     const uint32_t a = tmem + (buf ? C::COL_S1 : C::COL_S0);
                     const uint64_t bd = vdesc0 + (uint64_t)((vslot * C::TILE_BYTES) >> 4);
+                    // split rows: the P of column half h sits at columns 64 h .. 64 h + 31
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)
-                        umma_ts(d, a + ks * 8, bd + (uint64_t)((ks * 2048) >> 4), IDESC_O, (!first) || ks > 0);
+                        umma_ts(d, a + (C::NSPLIT == 2 ? (ks / 4) * 64 + (ks % 4) * 8 : ks * 8), bd + (uint64_t)((ks * 2048) >> 4),
+                                IDESC_O, (!first) || ks > 0);
                 }
             };
             auto commit = [&](uint64_t* bar) {
                 if (elect_one()) umma_commit(smem_u32(bar));
             };
+            // a ring stage goes back to the producer once the MMAs issued so far have completed
+            auto release_tile = [&](int slot) { commit(&ctl.kv_empty[slot]); };
+            // wait for the next tile of the ring
             auto wait_kv = [&](int& slot, int where, int item) -> bool {
                 slot = (int)(nuse % C::NSTAGE);
                 if (!ctl_wait(&ctl.kv_full[slot], (uint32_t)((nuse / C::NSTAGE) & 1), &ctl)) {
@@ -492,22 +525,28 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if constexpr (NQ == 2) {
                     issue_s(0, 0, slot); commit(&ctl.s_full[0]);
                     issue_s(1, 1, slot); commit(&ctl.s_full[1]);
-                    commit(&ctl.kv_empty[slot]);
+                    release_tile(slot);
                 } else {
                     issue_s(0, gs & 1, slot);
                     commit(&ctl.s_full[gs & 1]);
-                    commit(&ctl.kv_empty[slot]);
+                    release_tile(slot);
                     ++gs;
                 }
                 bool first = true;
                 while (cur >= 0) {
                     const int nxt = walk.next();
                     int vslot, kslot = 0;
-                    if (!wait_kv(vslot, 22, (int)item)) { ok = false; break; }
+                    // the ring order of K(next) and V(current) is the producer's
+                    if constexpr (!C::K_AHEAD) {
+                        if (!wait_kv(vslot, 22, (int)item)) { ok = false; break; }
+                    }
                     if (nxt >= 0) {
                         if (!wait_kv(kslot, 23, (int)item)) { ok = false; break; }
                     } else {
                         commit(&ctl.q_empty);     // every S of this item has been issued
+                    }
+                    if constexpr (C::K_AHEAD) {
+                        if (!wait_kv(vslot, 22, (int)item)) { ok = false; break; }
                     }
                     if constexpr (NQ == 2) {
                         // query tile 0
@@ -522,10 +561,10 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         ++np[1];
                         tc_fence_after();
                         issue_o(1, 1, vslot, first);
-                        commit(&ctl.kv_empty[vslot]);
+                        release_tile(vslot);
                         if (nxt >= 0) {
                             issue_s(1, 1, kslot); commit(&ctl.s_full[1]);
-                            commit(&ctl.kv_empty[kslot]);
+                            release_tile(kslot);
                         } else {
                             commit(&ctl.o_full[1]);
                         }
@@ -534,7 +573,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         if (nxt >= 0) {
                             issue_s(0, gs & 1, kslot);
                             commit(&ctl.s_full[gs & 1]);
-                            commit(&ctl.kv_empty[kslot]);
+                            release_tile(kslot);
                             ++gs;
                         }
                         const int buf = gp & 1;
@@ -542,7 +581,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         ++gp;
                         tc_fence_after();
                         issue_o(0, buf, vslot, first);
-                        commit(&ctl.kv_empty[vslot]);
+                        release_tile(vslot);
                         commit(&ctl.pv_done);
                         if (nxt < 0) commit(&ctl.o_full[0]);
                     }
@@ -555,11 +594,15 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         __syncwarp();
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ softmax + epilogue
-        if constexpr (NQ == 2) reg_inc<REGS_SOFTMAX_2WG>(); else reg_inc<REGS_SOFTMAX_1WG>();
-        const int x = (warp - 4) >> 2;                       // query tile of this warpgroup (0 when NQ == 1)
+        reg_inc<REGS_SOFTMAX_2WG>();
+        constexpr int NSPLIT = C::NSPLIT, NC = C::NC;
+        const int wg = (warp - 4) >> 2;
+        const int x = NSPLIT == 2 ? 0 : wg;                  // query tile of this warpgroup
+        const int half = NSPLIT == 2 ? wg : 0;               // split rows: its column half of every key tile
         const int row_in_tile = ((warp & 3) << 5) | lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t t_o = tmem + lane_base + (x ? C::COL_O1 : C::COL_O0);
+        const uint32_t t_o = tmem + lane_base + (x ? C::COL_O1 : C::COL_O0) + half * (D / 2);   // its part of the O row
+        uint32_t nx = 0;                                     // split rows: exchanges done with the partner half
         // logits in log2 units: sl2 * S, or with a softcap sl2 * tanh(cap_in * S)
         const float sl2 = SOFTCAP ? p.softcap * LOG2E : p.scale * LOG2E;
         const float cap_in = SOFTCAP ? p.scale / p.softcap : 0.f;
@@ -604,36 +647,48 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 const int buf = NQ == 2 ? x : (int)(ns & 1);
                 const uint32_t par = NQ == 2 ? (ns & 1) : ((ns >> 1) & 1);
                 if (!ctl_wait(&ctl.s_full[buf], par, &ctl)) { report_timeout(p, &ctl, 30 + x, (int)item); ok = false; break; }
-                const uint32_t t_s = tmem + lane_base + (buf ? C::COL_S1 : C::COL_S0);
+                // this thread's NC S columns; its packed P columns overwrite the first half of them
+                const uint32_t t_s = tmem + lane_base + (buf ? C::COL_S1 : C::COL_S0) + half * NC;
                 tc_fence_after();
-                uint32_t pk[64];
+                uint32_t pk[NC / 2];
                 if (tm.all_masked) {
 #pragma unroll
-                    for (int c = 0; c < 64; ++c) pk[c] = 0u;
+                    for (int c = 0; c < NC / 2; ++c) pk[c] = 0u;
                 } else {
-                    uint32_t sr[128];
+                    uint32_t sr[NC];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) tmem_ld32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[c * 32]));
+                    for (int c = 0; c < NC / 32; ++c) tmem_ld32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[c * 32]));
                     tmem_wait_ld();
                     if (SOFTCAP) {
 #pragma unroll
-                        for (int c = 0; c < 128; ++c) sr[c] = __float_as_uint(tanh_approx(__uint_as_float(sr[c]) * cap_in));
+                        for (int c = 0; c < NC; ++c) sr[c] = __float_as_uint(tanh_approx(__uint_as_float(sr[c]) * cap_in));
                     }
                     if (tm.masked) {
 #pragma unroll
-                        for (int c = 0; c < 128; ++c)
-                            sr[c] = ((tm.kw[c >> 5] >> (c & 31)) & 1u) ? sr[c] : 0xff800000u;      // -inf
+                        for (int c = 0; c < NC; ++c)
+                            sr[c] = ((tm.kw[(NSPLIT == 2 ? half * 2 : 0) + (c >> 5)] >> (c & 31)) & 1u) ? sr[c] : 0xff800000u;      // -inf
                     }
                     // ---- row maximum of the tile: four independent chains of three-input maxima
                     float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                    for (int c = 0; c < 128; c += 8) {
+                    for (int c = 0; c < NC; c += 8) {
                         mx0 = max3(mx0, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
                         mx1 = max3(mx1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
                         mx2 = max3(mx2, __uint_as_float(sr[c + 4]), __uint_as_float(sr[c + 5]));
                         mx3 = max3(mx3, __uint_as_float(sr[c + 6]), __uint_as_float(sr[c + 7]));
                     }
-                    const float mt = max3(mx0, mx1, fmaxf(mx2, mx3)) * sl2;   // log2 units (sl2 > 0; -inf stays -inf)
+                    float mraw = max3(mx0, mx1, fmaxf(mx2, mx3));
+                    if constexpr (NSPLIT == 2) {
+                        // the two threads of a row exchange the maxima of their halves and then take the same decisions
+                        const int par = (int)(nx & 1);
+                        xval(par, half, row_in_tile) = mraw;
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&ctl.xchg[warp & 3]));
+                        if (!ctl_wait(&ctl.xchg[warp & 3], (uint32_t)par, &ctl)) { report_timeout(p, &ctl, 36, (int)item); ok = false; }
+                        mraw = fmaxf(mraw, xval(par, half ^ 1, row_in_tile));
+                        ++nx;
+                    }
+                    const float mt = mraw * sl2;                     // log2 units (sl2 > 0; -inf stays -inf)
                     // ---- lazy maximum: raise the reference only when it lags by more than the threshold
                     float factor = 1.f;
                     bool raise = false;
@@ -652,7 +707,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         if (!pv_ok) { report_timeout(p, &ctl, 35, (int)item); ok = false; }
                         tc_fence_after();
 #pragma unroll 1
-                        for (int c = 0; c < D / 16; ++c) {
+                        for (int c = 0; c < D / 16 / NSPLIT; ++c) {      // this thread's part of the O row
                             uint32_t ov[16];
                             tmem_ld16(t_o + c * 16, ov);
                             tmem_wait_ld();
@@ -669,7 +724,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
                     for (int e = 0; e < 4; ++e) acc[e] = make_float2(0.f, 0.f);
 #pragma unroll
-                    for (int c = 0; c < 128; c += 8) {
+                    for (int c = 0; c < NC; c += 8) {
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const float2 xv = __ffma2_rn(make_float2(__uint_as_float(sr[c + 2 * e]),
@@ -687,8 +742,8 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     }
                     l += (acc[0].x + acc[0].y) + (acc[1].x + acc[1].y) + ((acc[2].x + acc[2].y) + (acc[3].x + acc[3].y));
                 }
-                tmem_st32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
-                tmem_st32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+#pragma unroll
+                for (int c = 0; c < NC / 64; ++c) tmem_st32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[c * 32]));
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&ctl.p_full[buf]));
@@ -698,12 +753,23 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
             if (!ok) break;
             // ---- epilogue: O / l -> bf16 -> global, lse
+            if constexpr (NSPLIT == 2) {
+                // the two halves add their row sums
+                const int par = (int)(nx & 1);
+                xval(par, half, row_in_tile) = l;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl.xchg[warp & 3]));
+                if (!ctl_wait(&ctl.xchg[warp & 3], (uint32_t)par, &ctl)) { report_timeout(p, &ctl, 38, (int)item); break; }
+                l += xval(par, half ^ 1, row_in_tile);
+                ++nx;
+            }
             if (!ctl_wait(&ctl.o_full[x], it & 1, &ctl)) { report_timeout(p, &ctl, 40 + x, (int)item); break; }
             tc_fence_after();
             const float inv_l = 1.f / l;
-            __nv_bfloat16* orow = p.o + (size_t)bb * p.o_sb + (size_t)h * p.o_sh + (size_t)(valid ? i : 0) * p.o_sn;
+            __nv_bfloat16* orow = p.o + (size_t)bb * p.o_sb + (size_t)h * p.o_sh + (size_t)(valid ? i : 0) * p.o_sn +
+                                  half * (D / 2);
 #pragma unroll 1
-            for (int c = 0; c < D / 32; ++c) {
+            for (int c = 0; c < D / 32 / NSPLIT; ++c) {
                 uint32_t ov[32];
                 tmem_ld32(t_o + c * 32, ov);
                 tmem_wait_ld();
@@ -719,7 +785,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     }
                 }
             }
-            if (valid) p.lse[(size_t)hq * p.n + i] = (m_used + lg2_approx(l)) * LN2;
+            if (valid && half == 0) p.lse[(size_t)hq * p.n + i] = (m_used + lg2_approx(l)) * LN2;
             tc_fence_before();
             ++it;
         }
