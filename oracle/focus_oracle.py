@@ -32,6 +32,15 @@ Passages of the paper each function follows:
                         combined with Appendix C's mask (same-class-sharing keys up to the block's last
                         position; other keys only inside the window).
 
+* ``router_scores``     Sec. 2 "Learned grouping", the argument of Eq. 1's normalisation: (W_g h_i) . C_g.
+* ``sinkhorn``          Sec. 2 "Learned grouping", the two-step Sinkhorn normalisation: exponentiate the scores
+                        over the temperature, then N times divide by the sums over tokens and by the sums over
+                        groups, in that order.
+* ``gated_attn``        Sec. 2 "Gated attention" (Eq. 2), the training-time forward over all causal pairs: the
+                        score of a distant pair is multiplied by sigmoid(lambda g_i . g_j), a pair inside the
+                        window keeps its score.  The equation is followed as printed, so the gate of two
+                        orthogonal assignments is sigmoid(0) = 1/2 (the prose around it says "towards zero").
+
 Parity status: every function above is pinned by the CPU tests.  "parity unpinned": the paper's
 perplexity and benchmark numbers (datasets and trained weights are not available).
 """
@@ -369,3 +378,54 @@ def assign_hidden(h_bits: np.ndarray, Wg: np.ndarray, C: np.ndarray, topk: int, 
     srt = np.take_along_axis(S, order, axis=1)
     margins = srt[:, topk - 1] - srt[:, topk] if topk < K else np.full(n, np.inf)
     return masks, margins
+
+
+def router_scores(h_bits: np.ndarray, Wg: np.ndarray, C: np.ndarray) -> np.ndarray:
+    """S[i, g] = <Wg^T h_i, C_g> in fp64: project the hidden state, then score it against the centroids."""
+    Z = bf16_bits_to_f64(np.asarray(h_bits)) @ np.asarray(Wg, np.float64)
+    return Z @ np.asarray(C, np.float64).T
+
+
+def sinkhorn(S: np.ndarray, tau: float, iters: int) -> np.ndarray:
+    """Sinkhorn normalisation of scores S [n, K] at temperature tau: the soft assignments g [n, K].
+
+    Step 1: Q = exp(S / tau).  Step 2, ``iters`` times: divide every column by its sum over the tokens, then
+    every row by its sum over the groups.
+    """
+    Q = np.exp(np.asarray(S, np.float64) / float(tau))
+    for _ in range(int(iters)):
+        Q = Q / Q.sum(axis=0, keepdims=True)
+        Q = Q / Q.sum(axis=1, keepdims=True)
+    return Q
+
+
+def gated_attn(q_bits, k_bits, v_bits, g, lam, window, scale=None, rows=None):
+    """Training-time gated attention forward over all causal pairs.
+
+    q_bits uint16 [Hq, n, D], k_bits / v_bits uint16 [Hkv, n, D] (bf16 bit patterns), g float [n, K] (one soft
+    assignment per token, shared by all heads), ``lam`` the gate sharpness, ``window`` the local window w.
+    For j <= i:  s_ij = scale * <q_i, k_j> * (1 if i - j <= w else sigmoid(lam * <g_i, g_j>)); row softmax.
+    Returns (O f64 [Hq, len(rows), D], lse f64 [Hq, len(rows)]); rows default to all.
+    """
+    Q = bf16_bits_to_f64(np.asarray(q_bits)); Kx = bf16_bits_to_f64(np.asarray(k_bits)); V = bf16_bits_to_f64(np.asarray(v_bits))
+    Hq, n, D = Q.shape
+    G = Hq // Kx.shape[0]
+    sc = 1.0 / np.sqrt(D) if scale is None else float(scale)
+    g = np.asarray(g, np.float64)
+    rows = np.arange(n) if rows is None else np.asarray(rows, np.int64)
+    O = np.zeros((Hq, rows.size, D)); lse = np.zeros((Hq, rows.size))
+    j = np.arange(n)
+    for r, i in enumerate(rows):
+        aff = g @ g[i]                                          # g_i . g_j for every j
+        local = (i - j) <= window
+        factor = np.where(local, 1.0, 1.0 / (1.0 + np.exp(-float(lam) * aff)))
+        causal = j <= i
+        for h in range(Hq):
+            s = sc * (Kx[h // G] @ Q[h, i]) * factor
+            s = s[causal]
+            m = s.max()
+            e = np.exp(s - m)
+            Z = e.sum()
+            O[h, r] = (e / Z) @ V[h // G][causal]
+            lse[h, r] = m + np.log(Z)
+    return O, lse

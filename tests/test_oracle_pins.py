@@ -454,3 +454,98 @@ def test_bias_is_the_inference_residue_of_sinkhorn_column_scaling():
     mass = Q.sum(axis=0)                     # Sinkhorn did balance the groups' mass; the plain row softmax does not
     P = np.exp(S / tau); P /= P.sum(axis=1, keepdims=True)
     assert mass.max() / mass.min() < 0.5 * P.sum(axis=0).max() / P.sum(axis=0).min()
+
+
+# ---------------------------------------------------------------- training-time forward: Sinkhorn and the soft gate (Sec. 2)
+def test_router_scores_hand_case():
+    """d = 2, d_g = 2, K = 2 in small integers, worked by hand: z = h Wg, S = z C^T"""
+    h = bits(np.array([[1., 2.], [3., -1.]]))
+    Wg = np.array([[1., 0.], [2., 1.]])            # z_0 = (1 + 4, 2) = (5, 2);  z_1 = (3 - 2, -1) = (1, -1)
+    C = np.array([[1., 1.], [0., -2.]])            # S_0 = (7, -4);  S_1 = (0, 2)
+    np.testing.assert_array_equal(fo.router_scores(h, Wg, C), np.array([[7., -4.], [0., 2.]]))
+
+
+def test_sinkhorn_hand_2x2():
+    """exp(S / tau) = [[1, 2], [3, 4]]; two iterations worked by hand in fractions.
+    It. 1: column sums 4, 6 -> [[1/4, 1/3], [3/4, 2/3]]; row sums 7/12, 17/12 -> [[3/7, 4/7], [9/17, 8/17]].
+    It. 2: column sums 114/119, 124/119 -> [[17/38, 17/31], [21/38, 14/31]]; row sums 1173/1178, 1183/1178
+           -> [[31/69, 38/69], [93/169, 76/169]]."""
+    tau = 0.7
+    S = tau * np.log(np.array([[1., 2.], [3., 4.]]))
+    np.testing.assert_allclose(fo.sinkhorn(S, tau, 1), [[3 / 7, 4 / 7], [9 / 17, 8 / 17]], rtol=1e-14)
+    np.testing.assert_allclose(fo.sinkhorn(S, tau, 2), [[31 / 69, 38 / 69], [93 / 169, 76 / 169]], rtol=1e-14)
+    # rows first, columns second (the wrong order) gives [[1/3, 2/3], [3/7, 4/7]] -> columns ... : not the values above
+    assert abs(fo.sinkhorn(S, tau, 1)[0, 0] - (1 / 3) / (1 / 3 + 3 / 7)) > 1e-3
+
+
+def test_sinkhorn_2x2_limit_closed_form():
+    """Two tokens, two groups: the doubly stochastic scaling of [[a, b], [c, d]] is [[x, 1-x], [1-x, x]] with
+    x = sqrt(ad) / (sqrt(ad) + sqrt(bc)) (diagonal scalings keep the cross ratio ad / bc)."""
+    a, b, c, d = 1., 2., 3., 4.
+    x = math.sqrt(a * d) / (math.sqrt(a * d) + math.sqrt(b * c))
+    got = fo.sinkhorn(np.log(np.array([[a, b], [c, d]])), 1.0, 300)
+    np.testing.assert_allclose(got, [[x, 1 - x], [1 - x, x]], rtol=1e-12)
+
+
+def test_sinkhorn_invariants():
+    rng = np.random.default_rng(5)
+    n, K, tau = 400, 8, 0.5
+    S = rng.standard_normal((n, K))
+    g = fo.sinkhorn(S, tau, 10)
+    np.testing.assert_allclose(g.sum(axis=1), 1.0, atol=1e-14)           # the last step normalises the rows
+    assert np.all(g > 0)
+    np.testing.assert_allclose(fo.sinkhorn(S, tau, 200).sum(axis=0), n / K, rtol=1e-9)   # balanced groups at convergence
+    # a per-group offset of the scores is removed by the first division over the tokens
+    np.testing.assert_allclose(fo.sinkhorn(S + rng.standard_normal(K)[None, :], tau, 10), g, rtol=1e-11)
+    # a per-token offset is not (finite number of iterations): the order of the two divisions matters
+    assert np.abs(fo.sinkhorn(S + rng.standard_normal(n)[:, None], tau, 1) - fo.sinkhorn(S, tau, 1)).max() > 1e-3
+    # one group: everything belongs to it; equal scores: equal shares
+    np.testing.assert_array_equal(fo.sinkhorn(S[:, :1], tau, 10), np.ones((n, 1)))
+    np.testing.assert_allclose(fo.sinkhorn(np.full((n, K), 0.3), tau, 10), 1.0 / K, rtol=1e-14)
+    # one token: the division over tokens makes every entry 1, the division over groups 1/K
+    np.testing.assert_allclose(fo.sinkhorn(S[:1], tau, 3), np.full((1, K), 1.0 / K), rtol=1e-14)
+
+
+def test_gated_attn_hand_case():
+    """n = 3, D = 1, K = 2, w = 0, lambda = ln 3, scale = ln 2, worked by hand.
+    g = (e0, e1, e0): sigmoid(lambda * 1) = 3/4, sigmoid(0) = 1/2.  q = (1, 1, 2), k = (2, 4, 1), v = (7, 14, 21).
+    Row 0: s = 2 ln2 -> o = 7, lse = ln 4.
+    Row 1: s_10 = 1*2*ln2 * 1/2 = ln 2 -> 2;  s_11 = 4 ln 2 -> 16;  o = (2*7 + 16*14) / 18 = 119/9, lse = ln 18.
+    Row 2: s_20 = 2*2*ln2 * 3/4 = 3 ln 2 -> 8;  s_21 = 2*4*ln2 * 1/2 = 4 ln 2 -> 16;  s_22 = 2 ln 2 -> 4;
+           o = (8*7 + 16*14 + 4*21) / 28 = 13, lse = ln 28."""
+    q = bits(np.array([[[1.], [1.], [2.]]])); k = bits(np.array([[[2.], [4.], [1.]]])); v = bits(np.array([[[7.], [14.], [21.]]]))
+    g = np.array([[1., 0.], [0., 1.], [1., 0.]])
+    O, lse = fo.gated_attn(q, k, v, g, math.log(3.0), 0, scale=math.log(2.0))
+    np.testing.assert_allclose(O[0, :, 0], [7.0, 119.0 / 9.0, 13.0], rtol=1e-13)
+    np.testing.assert_allclose(lse[0], np.log([4.0, 18.0, 28.0]), rtol=1e-13)
+    # window 1 makes (1,0) and (2,1) local: row 1 -> (4*7 + 16*14)/20, row 2 -> (8*7 + 256*14 + 4*21)/268
+    O, lse = fo.gated_attn(q, k, v, g, math.log(3.0), 1, scale=math.log(2.0))
+    np.testing.assert_allclose(O[0, :, 0], [7.0, 252.0 / 20.0, 3724.0 / 268.0], rtol=1e-13)
+
+
+def test_gated_attn_reduces_to_library_attention():
+    rng = np.random.default_rng(11)
+    Hq, Hkv, n, D, K = 4, 2, 96, 16, 4
+    qb, kb, vb = rand_bits(rng, (Hq, n, D)), rand_bits(rng, (Hkv, n, D)), rand_bits(rng, (Hkv, n, D))
+    g = fo.sinkhorn(rng.standard_normal((n, K)), 0.5, 10)
+    ref = sdpa_causal(qb, kb, vb, 1.0 / math.sqrt(D))
+    # the window covers the whole sequence: the gate never applies
+    O, _ = fo.gated_attn(qb, kb, vb, g, 7.0, n, None)
+    np.testing.assert_allclose(O, ref, atol=1e-12)
+    # every token wholly in one group and a sharp gate: sigmoid(60) = 1 to 1e-26
+    one = np.zeros((n, K)); one[:, 2] = 1.0
+    O, _ = fo.gated_attn(qb, kb, vb, one, 60.0, 3, None)
+    np.testing.assert_allclose(O, ref, atol=1e-12)
+
+
+def test_gated_attn_half_gate_is_half_scale():
+    """g = 0 gives the gate sigmoid(0) = 1/2 on every distant pair.  With w = 0 only the diagonal is local, and
+    with k_i orthogonal to q_i the diagonal logit is 0 at any scale: the result is library attention at half
+    the scale."""
+    rng = np.random.default_rng(12)
+    H, n = 3, 64
+    q = rng.integers(-4, 5, size=(H, n, 2)).astype(np.float64)
+    k = np.stack([-q[..., 1], q[..., 0]], axis=-1) * rng.integers(1, 3, size=(H, n, 1))
+    qb, kb, vb = bits(q), bits(k), rand_bits(rng, (H, n, 2))
+    O, _ = fo.gated_attn(qb, kb, vb, np.zeros((n, 4)), 5.0, 0, scale=0.25)
+    np.testing.assert_allclose(O, sdpa_causal(qb, kb, vb, 0.125), atol=1e-12)
