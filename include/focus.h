@@ -260,6 +260,48 @@ FOCUS_API int focus_count_kept_noalloc(const focus_shape* shape, const uint32_t*
                                        unsigned long long* counts_out, void* stream);
 
 /*
+ * Training-time forward (paper Sec. 2 "Learned grouping" and "Gated attention", Eq. 1 and Eq. 2).  During
+ * training nothing is pruned: every causal pair is computed and the score of a distant pair is multiplied by a
+ * gate built from soft group assignments, so this path has no speedup over dense attention (the paper says so).
+ *
+ * focus_router_scores -- S[b, i, g] = (W_g h_i) . C_g, the argument of Eq. 1's normalisation, in fp32 on the
+ * exact bf16 hidden states.  Arguments as for focus_assign_hidden;
+ *   scores_out  device fp32 [batch, n, ld], ld = 4 for K <= 4, else 8 for K <= 8, else 16 or 32 (the smallest
+ *               that holds K); entries g >= K are written as 0.  16-byte aligned.
+ *
+ * focus_sinkhorn -- the Sinkhorn normalisation of Sec. 2: Q = exp(S / tau); `iters` times divide every column
+ * by its sum over the tokens of the sequence, then every row by its sum over the groups.  Each sequence of the
+ * batch is normalised on its own.  Computed in the log domain (offsets per token and per group, fp32, column
+ * sums accumulated in fp64), which is the same arithmetic without overflow; after the first row division every
+ * entry lies in (0, 1].
+ *   shape       batch, n, K are read             scores   device fp32 [batch, n, ld] (ld as above)
+ *   tau > 0, iters >= 1 (the paper uses tau = 0.1, iters = 10)
+ *   ws          device scratch, focus_sinkhorn_workspace_bytes(shape, iters) bytes, 16-byte aligned
+ *   g_out       device fp32 [batch, n, ld]; entries g >= K are written as 0; may be the scores buffer itself
+ *
+ * focus_gate_attn_fwd -- Eq. 2: for j <= i
+ *        s_ij = scale * q_i.k_j * ( 1 if i - j <= window, else sigmoid(lambda * g_i.g_j) ),
+ * then exact row softmax over all j <= i, o_i = sum_j p_ij v_j, lse_i = log sum_j exp(s_ij).  The equation is
+ * followed as printed: two orthogonal assignments give the gate sigmoid(0) = 1/2.  Same kernel, operand
+ * precision and accumulation as focus_attn_fwd in dense causal mode; the gate is evaluated in fp32 as
+ * 1/2 + 1/2 tanh(lambda/2 g_i.g_j) with the hardware tanh approximation.
+ *   shape       softcap must be 0; K <= 8 (FOCUS_ERR_UNSUPPORTED otherwise); masks and topk are not used
+ *   q, k, v, o, lse, dev_status   as for focus_attn_fwd
+ *   g           device fp32 [batch, n, ld], ld = 4 (K <= 4) or 8; one assignment per token, shared by all heads;
+ *               entries g >= K must be 0 (focus_sinkhorn writes them so); 16-byte aligned
+ */
+FOCUS_API int focus_router_scores(const focus_shape* shape, const void* h, int64_t stride_b, int64_t stride_n,
+                                  int32_t d_model, int32_t d_g, const float* Wg, const float* C, float* folded,
+                                  float* scores_out, void* stream);
+FOCUS_API int32_t focus_soft_ld(int32_t K);     /* the row length ld for K groups (4, 8, 16 or 32; 0 if K is out of range) */
+FOCUS_API size_t focus_sinkhorn_workspace_bytes(const focus_shape* shape, int32_t iters);
+FOCUS_API int focus_sinkhorn(const focus_shape* shape, const float* scores, float tau, int32_t iters, void* ws,
+                             size_t ws_bytes, float* g_out, void* stream);
+FOCUS_API int focus_gate_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k, focus_tensor v,
+                                  const float* g, float lambda, focus_tensor o, float* lse, int32_t* dev_status,
+                                  void* stream);
+
+/*
  * focus_selftest_umma -- diagnostic, not on the hot path (the paper has no counterpart): one
  * 128 x 128 x D tile S = A B^T and one 128 x D x 128 tile O = P V through the same TMA, descriptor
  * and tcgen05 building blocks as focus_attn_fwd, so that an encoding mistake shows up in isolation.

@@ -81,6 +81,16 @@ def lib():
         L.focus_decode_workspace_bytes.argtypes = [SP]
         L.focus_decode_step.restype = C.c_int
         L.focus_decode_step.argtypes = [SP, focus_tensor, focus_tensor, focus_tensor, vp, vp, focus_tensor, vp, vp, sz, vp]
+        L.focus_router_scores.restype = C.c_int
+        L.focus_router_scores.argtypes = [SP, vp, C.c_int64, C.c_int64, i32, i32, vp, vp, vp, vp, vp]
+        L.focus_soft_ld.restype = i32
+        L.focus_soft_ld.argtypes = [i32]
+        L.focus_sinkhorn_workspace_bytes.restype = sz
+        L.focus_sinkhorn_workspace_bytes.argtypes = [SP, i32]
+        L.focus_sinkhorn.restype = C.c_int
+        L.focus_sinkhorn.argtypes = [SP, vp, f32, i32, vp, sz, vp, vp]
+        L.focus_gate_attn_fwd.restype = C.c_int
+        L.focus_gate_attn_fwd.argtypes = [SP, focus_tensor, focus_tensor, focus_tensor, vp, f32, focus_tensor, vp, vp, vp]
         L.focus_count_kept.restype = C.c_int
         L.focus_count_kept.argtypes = [SP, vp, vp, vp, vp]
         L.focus_count_kept_noalloc.restype = C.c_int
@@ -174,6 +184,34 @@ def focus_decode_step(shape, q, k, v, mq_new, mk, o, lse, ws, stream=None):
         return focus_tensor(t.data_ptr(), t.stride(0), t.stride(1), t.shape[-1])
     _check(lib().focus_decode_step(C.byref(shape), vec_arg(q), tensor_arg(k), tensor_arg(v), _p(mq_new), _p(mk), vec_arg(o),
                                    _p(lse), _p(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def focus_soft_ld(K) -> int:
+    return int(lib().focus_soft_ld(K))
+
+
+def focus_router_scores(shape, h, Wg, Cg, folded, scores_out, stream=None):
+    """h bf16 [batch, n, d_model] (or [n, d_model]); scores_out fp32 [batch, n, focus_soft_ld(K)]"""
+    assert h.is_cuda and h.dtype == torch.bfloat16 and h.stride(-1) == 1
+    sb, sn = (h.stride(0), h.stride(1)) if h.dim() == 3 else (h.stride(0) * h.shape[0], h.stride(0))
+    _check(lib().focus_router_scores(C.byref(shape), _p(h), sb, sn, h.shape[-1], Wg.shape[1], _p(Wg), _p(Cg), _p(folded),
+                                     _p(scores_out), _stream(stream)))
+
+
+def focus_sinkhorn_workspace_bytes(shape, iters) -> int:
+    return int(lib().focus_sinkhorn_workspace_bytes(C.byref(shape), iters))
+
+
+def focus_sinkhorn(shape, scores, tau, iters, ws, g_out, stream=None):
+    """scores, g_out fp32 [batch, n, focus_soft_ld(K)] (may be the same tensor); ws uint8 scratch"""
+    _check(lib().focus_sinkhorn(C.byref(shape), _p(scores), tau, iters, _p(ws), ws.numel() * ws.element_size(), _p(g_out),
+                                _stream(stream)))
+
+
+def focus_gate_attn_fwd(shape, q, k, v, g, lam, o, lse, dev_status=None, stream=None):
+    """training-time gated forward; g fp32 [batch, n, focus_soft_ld(K)]"""
+    _check(lib().focus_gate_attn_fwd(C.byref(shape), tensor_arg(q), tensor_arg(k), tensor_arg(v), _p(g), lam, tensor_arg(o),
+                                     _p(lse), _p(dev_status), _stream(stream)))
 
 
 def focus_count_kept(shape, mq, tiles_ws, counts_out, stream=None):

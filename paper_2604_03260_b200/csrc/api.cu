@@ -192,7 +192,45 @@ int focus_assign_hidden(const focus_shape* shape, const void* h, int64_t stride_
         return fail(FOCUS_ERR_INVALID_ARG, "h and folded must be 16-byte aligned, strides multiples of 8 elements, stride_n >= d_model");
     if ((rc = require_sm100())) return rc;
     return launch_assign_hidden(shape, h, stride_b, stride_n, d_model, d_g, Wg, C, bias, folded, mq_out, mk_out, near_ties,
-                                near_tie_eps, (cudaStream_t)stream);
+                                near_tie_eps, nullptr, (cudaStream_t)stream);
+}
+
+int32_t focus_soft_ld(int32_t K) {
+    if (K < 1 || K > 32) return 0;
+    return K <= 4 ? 4 : (K <= 8 ? 8 : (K <= 16 ? 16 : 32));
+}
+
+int focus_router_scores(const focus_shape* shape, const void* h, int64_t stride_b, int64_t stride_n, int32_t d_model,
+                        int32_t d_g, const float* Wg, const float* C, float* folded, float* scores_out, void* stream) {
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if (!h || !Wg || !C || !folded || !scores_out) return fail(FOCUS_ERR_INVALID_ARG, "h, Wg, C, folded or scores_out is NULL");
+    if (d_model < 8 || d_model % 8 || d_g < 1) return fail(FOCUS_ERR_INVALID_ARG, "d_model must be a positive multiple of 8 and d_g >= 1");
+    if ((uintptr_t)h % 16 || (uintptr_t)folded % 16 || (uintptr_t)scores_out % 16 || stride_n % 8 || stride_b % 8 || stride_n < d_model)
+        return fail(FOCUS_ERR_INVALID_ARG,
+                    "h, folded and scores_out must be 16-byte aligned, strides multiples of 8 elements, stride_n >= d_model");
+    if ((rc = require_sm100())) return rc;
+    return launch_assign_hidden(shape, h, stride_b, stride_n, d_model, d_g, Wg, C, nullptr, folded, nullptr, nullptr, nullptr, 0.f,
+                                scores_out, (cudaStream_t)stream);
+}
+
+size_t focus_sinkhorn_workspace_bytes(const focus_shape* shape, int32_t iters) {
+    if (validate_shape(shape) || iters < 1) return 0;
+    return sinkhorn_workspace_bytes(shape, iters);
+}
+
+int focus_sinkhorn(const focus_shape* shape, const float* scores, float tau, int32_t iters, void* ws, size_t ws_bytes,
+                   float* g_out, void* stream) {
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if (!scores || !ws || !g_out) return fail(FOCUS_ERR_INVALID_ARG, "scores, ws or g_out is NULL");
+    if (!(tau > 0.f) || iters < 1 || iters > 1000) return fail(FOCUS_ERR_INVALID_ARG, "tau must be positive and iters in [1, 1000]");
+    if ((uintptr_t)scores % 16 || (uintptr_t)g_out % 16 || (uintptr_t)ws % 16)
+        return fail(FOCUS_ERR_INVALID_ARG, "scores, g_out and ws must be 16-byte aligned");
+    if (ws_bytes < sinkhorn_workspace_bytes(shape, iters))
+        return fail(FOCUS_ERR_CAPACITY, "sinkhorn workspace has %zu bytes, %zu needed", ws_bytes, sinkhorn_workspace_bytes(shape, iters));
+    if ((rc = require_sm100())) return rc;
+    return launch_sinkhorn(shape, scores, tau, iters, ws, g_out, (cudaStream_t)stream);
 }
 
 int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, const uint32_t* mk, int32_t layout, void* ws,
@@ -270,6 +308,33 @@ int focus_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k, foc
     if (tiles_ws && (rc = layout_of(shape, layout, &a.L))) return rc;
     const char* impl = getenv("FOCUS_ATTN_IMPL");
     if (impl && !strcmp(impl, "simple")) return launch_attn_simple(a, (cudaStream_t)stream);
+    return launch_attn_sm100(a, (cudaStream_t)stream);
+}
+
+int focus_gate_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k, focus_tensor v, const float* g, float lambda,
+                        focus_tensor o, float* lse, int32_t* dev_status, void* stream) {
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if ((rc = validate_tensor("q", q, true)) || (rc = validate_tensor("k", k, true)) ||
+        (rc = validate_tensor("v", v, true)) || (rc = validate_tensor("o", o, true)))
+        return rc;
+    if (!lse || !g) return fail(FOCUS_ERR_INVALID_ARG, "lse or g is NULL");
+    if ((uintptr_t)g % 16) return fail(FOCUS_ERR_INVALID_ARG, "g is not 16-byte aligned");
+    if (shape->softcap > 0.f) return fail(FOCUS_ERR_UNSUPPORTED, "the gated forward takes no softcap");
+    if (shape->K > 8) return fail(FOCUS_ERR_UNSUPPORTED, "the gated forward supports K <= 8 (K = %d)", shape->K);
+    if ((rc = require_sm100())) return rc;
+    AttnArgs a;
+    a.s = *shape;
+    a.q = q; a.k = k; a.v = v; a.o = o;
+    a.mq = nullptr; a.mk = nullptr;
+    a.ws = nullptr;                        // every causal pair is computed
+    a.lse = lse;
+    a.dev_status = dev_status;
+    a.scale = shape->scale > 0.f ? shape->scale : 1.0f / sqrtf((float)shape->D);
+    memset(&a.L, 0, sizeof a.L);
+    a.gate_g = g;
+    a.gate_ld = focus_soft_ld(shape->K);
+    a.gate_lambda = lambda;
     return launch_attn_sm100(a, (cudaStream_t)stream);
 }
 

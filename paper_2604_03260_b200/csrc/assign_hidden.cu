@@ -29,7 +29,8 @@ template <int KMAX>
 __global__ void __launch_bounds__(AH_THREADS)
 assign_hidden_kernel(const __nv_bfloat16* __restrict__ h, int64_t stride_b, int64_t stride_n, int n, int d, int K, int topk,
                      const float* __restrict__ folded, const float* __restrict__ bias, int Hq, int Hkv,
-                     uint32_t* __restrict__ mq, uint32_t* __restrict__ mk, unsigned long long* near_ties, float eps) {
+                     uint32_t* __restrict__ mq, uint32_t* __restrict__ mk, unsigned long long* near_ties, float eps,
+                     float* __restrict__ scores) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     unsigned char* tile = smem_raw;                                           // [2][AH_THREADS][AH_ROWB]
     float* cs = reinterpret_cast<float*>(smem_raw + 2 * AH_THREADS * AH_ROWB);   // [2][KMAX][AH_CHUNK]
@@ -104,6 +105,16 @@ assign_hidden_kernel(const __nv_bfloat16* __restrict__ h, int64_t stride_b, int6
     float score[KMAX];
 #pragma unroll
     for (int g = 0; g < KMAX; ++g) score[g] = dot2[g].x + dot2[g].y + ((bias && g < K) ? __ldg(bias + g) : 0.f);
+    if (scores) {   // the scores themselves (training-time soft assignment), rows of KMAX floats, zero beyond K
+        if (in) {
+            float4* o = reinterpret_cast<float4*>(scores + ((size_t)b * n + tok) * KMAX);
+#pragma unroll
+            for (int c = 0; c < KMAX / 4; ++c)
+                o[c] = make_float4(4 * c < K ? score[4 * c] : 0.f, 4 * c + 1 < K ? score[4 * c + 1] : 0.f,
+                                   4 * c + 2 < K ? score[4 * c + 2] : 0.f, 4 * c + 3 < K ? score[4 * c + 3] : 0.f);
+        }
+        return;
+    }
     uint32_t taken = 0;
     float last = 0.f, next = 0.f;
     // topk picks, then one more to measure the margin; strict '>' keeps the lowest index on ties
@@ -130,27 +141,28 @@ assign_hidden_kernel(const __nv_bfloat16* __restrict__ h, int64_t stride_b, int6
 
 template <int KMAX>
 static int launch_k(const focus_shape* s, const void* h, int64_t sb, int64_t sn, int d, const float* folded, const float* bias,
-                    uint32_t* mq, uint32_t* mk, unsigned long long* near_ties, float eps, cudaStream_t st) {
+                    uint32_t* mq, uint32_t* mk, unsigned long long* near_ties, float eps, float* scores, cudaStream_t st) {
     const size_t smem = (size_t)2 * AH_THREADS * AH_ROWB + (size_t)2 * KMAX * AH_CHUNK * sizeof(float);
     auto kern = assign_hidden_kernel<KMAX>;
     int rc = check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
                         "cudaFuncSetAttribute(assign_hidden)");
     if (rc) return rc;
     kern<<<dim3(cdiv(s->n, AH_THREADS), s->batch), AH_THREADS, smem, st>>>(
-        reinterpret_cast<const __nv_bfloat16*>(h), sb, sn, s->n, d, s->K, s->topk, folded, bias, s->Hq, s->Hkv, mq, mk, near_ties, eps);
+        reinterpret_cast<const __nv_bfloat16*>(h), sb, sn, s->n, d, s->K, s->topk, folded, bias, s->Hq, s->Hkv, mq, mk, near_ties, eps,
+        scores);
     return check_cuda(cudaGetLastError(), "assign_hidden kernel launch");
 }
 
 int launch_assign_hidden(const focus_shape* s, const void* h, int64_t sb, int64_t sn, int d, int dg, const float* Wg,
                          const float* C, const float* bias, float* folded, uint32_t* mq, uint32_t* mk,
-                         unsigned long long* near_ties, float eps, cudaStream_t st) {
+                         unsigned long long* near_ties, float eps, float* scores, cudaStream_t st) {
     fold_router_kernel<<<dim3(cdiv(d, 256), s->K), 256, 0, st>>>(Wg, C, d, dg, s->K, folded);
     int rc = check_cuda(cudaGetLastError(), "fold_router kernel launch");
     if (rc) return rc;
-    if (s->K <= 4) return launch_k<4>(s, h, sb, sn, d, folded, bias, mq, mk, near_ties, eps, st);
-    if (s->K <= 8) return launch_k<8>(s, h, sb, sn, d, folded, bias, mq, mk, near_ties, eps, st);
-    if (s->K <= 16) return launch_k<16>(s, h, sb, sn, d, folded, bias, mq, mk, near_ties, eps, st);
-    return launch_k<32>(s, h, sb, sn, d, folded, bias, mq, mk, near_ties, eps, st);
+    if (s->K <= 4) return launch_k<4>(s, h, sb, sn, d, folded, bias, mq, mk, near_ties, eps, scores, st);
+    if (s->K <= 8) return launch_k<8>(s, h, sb, sn, d, folded, bias, mq, mk, near_ties, eps, scores, st);
+    if (s->K <= 16) return launch_k<16>(s, h, sb, sn, d, folded, bias, mq, mk, near_ties, eps, scores, st);
+    return launch_k<32>(s, h, sb, sn, d, folded, bias, mq, mk, near_ties, eps, scores, st);
 }
 
 }  // namespace focus

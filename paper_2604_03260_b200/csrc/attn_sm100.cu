@@ -103,6 +103,10 @@ struct AttnParams {
     const int32_t* qrange;
     const int32_t* order;
     const unsigned long long* counters;
+    // training-time soft gate (Sec. 2 "Gated attention"): assignments [B, n, gate_ld] fp32, lambda / 2
+    const float* gate_g;
+    int gate_ld;
+    float gate_hl;
 };
 
 // Enumerates the key tiles a 256-row query block visits, in increasing order.  Every role of the
@@ -345,7 +349,7 @@ __device__ __forceinline__ void build_tile_mask_sorted(TileMask& tm, int w, cons
     }
 }
 
-template <int D, bool SOFTCAP>
+template <int D, bool SOFTCAP, bool GATE>
 __global__ void __launch_bounds__(AttnCfg<D>::THREADS, 1)
 focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
@@ -634,6 +638,19 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             const int f_x = (!p.dense && dfar > 0) ? (int)(dfar / 128) : 0;   // tiles b < f_x are far for this query tile
             float m_used = -INFINITY, l = 0.f;
             bool first = true;
+            // soft gate: this row's assignment times lambda / 2 (sigmoid(x) = 1/2 + 1/2 tanh(x / 2))
+            float gi[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            if constexpr (GATE) {
+                if (valid) {
+                    const float4* gp = reinterpret_cast<const float4*>(p.gate_g + ((size_t)bb * p.n + (size_t)i) * p.gate_ld);
+                    const float4 g0 = __ldg(gp);
+                    gi[0] = g0.x * p.gate_hl; gi[1] = g0.y * p.gate_hl; gi[2] = g0.z * p.gate_hl; gi[3] = g0.w * p.gate_hl;
+                    if (p.gate_ld == 8) {
+                        const float4 g1 = __ldg(gp + 1);
+                        gi[4] = g1.x * p.gate_hl; gi[5] = g1.y * p.gate_hl; gi[6] = g1.z * p.gate_hl; gi[7] = g1.w * p.gate_hl;
+                    }
+                }
+            }
             for (; kb >= 0; kb = walk.next()) {
                 TileMask tm;
                 if (p.sorted) {
@@ -662,6 +679,29 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     if (SOFTCAP) {
 #pragma unroll
                         for (int c = 0; c < NC; ++c) sr[c] = __float_as_uint(tanh_approx(__uint_as_float(sr[c]) * cap_in));
+                    }
+                    if constexpr (GATE) {
+                        // Eq. 2: the score of a distant pair (i - j > w) is multiplied by sigmoid(lambda g_i . g_j).
+                        // The key assignments are read with warp-uniform addresses (one L1 line serves the warp).
+                        const long long j0 = (long long)kb * 128 + half * NC;
+                        const long long ifar = i - p.w;                   // columns j < ifar are distant for this row
+                        if (__any_sync(0xffffffffu, valid && ifar > j0)) {
+                            const float* gk = p.gate_g + (size_t)bb * p.n * p.gate_ld;
+                            const bool wide = p.gate_ld == 8;
+#pragma unroll
+                            for (int c = 0; c < NC; ++c) {
+                                const long long j = j0 + c;
+                                const float4* gp = reinterpret_cast<const float4*>(gk + (size_t)(j < p.n ? j : p.n - 1) * p.gate_ld);
+                                const float4 a0 = __ldg(gp);
+                                float aff = fmaf(gi[0], a0.x, fmaf(gi[1], a0.y, fmaf(gi[2], a0.z, gi[3] * a0.w)));
+                                if (wide) {
+                                    const float4 a1 = __ldg(gp + 1);
+                                    aff += fmaf(gi[4], a1.x, fmaf(gi[5], a1.y, fmaf(gi[6], a1.z, gi[7] * a1.w)));
+                                }
+                                const float gate = fmaf(tanh_approx(aff), 0.5f, 0.5f);
+                                if (j < ifar) sr[c] = __float_as_uint(__uint_as_float(sr[c]) * gate);
+                            }
+                        }
                     }
                     if (tm.masked) {
 #pragma unroll
@@ -796,7 +836,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
-template <int D, bool SOFTCAP>
+template <int D, bool SOFTCAP, bool GATE>
 static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
     using C = AttnCfg<D>;
     CUtensorMap tq, tk, tv;
@@ -846,11 +886,12 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
     p.qrange = sorted ? reinterpret_cast<const int32_t*>(a.ws + a.L.qrange) : nullptr;
     p.order = sorted ? reinterpret_cast<const int32_t*>(a.ws + a.L.order) : nullptr;
     p.counters = a.ws ? reinterpret_cast<const unsigned long long*>(a.ws + a.L.counters) : nullptr;
+    p.gate_g = a.gate_g; p.gate_ld = a.gate_ld; p.gate_hl = 0.5f * a.gate_lambda;
     if (sorted) p.nitems = (long long)a.s.batch * a.s.Hq * p.nqblk * p.ipb;
     int dev = 0, sms = 0;
     if ((rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice"))) return rc;
     if ((rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "cudaDeviceGetAttribute"))) return rc;
-    auto kern = focus_attn_kernel<D, SOFTCAP>;
+    auto kern = focus_attn_kernel<D, SOFTCAP, GATE>;
     if ((rc = check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES),
                          "cudaFuncSetAttribute(attn)")))
         return rc;
@@ -861,10 +902,17 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
 
 int launch_attn_sm100(const AttnArgs& a, cudaStream_t st) {
     const bool cap = a.s.softcap > 0.f;
+    if (a.gate_g) {      // training-time gated forward: dense causal walk, no softcap
+        switch (a.s.D) {
+            case 64: return launch_attn_t<64, false, true>(a, st);
+            case 128: return launch_attn_t<128, false, true>(a, st);
+            case 256: return launch_attn_t<256, false, true>(a, st);
+        }
+    }
     switch (a.s.D) {
-        case 64: return cap ? launch_attn_t<64, true>(a, st) : launch_attn_t<64, false>(a, st);
-        case 128: return cap ? launch_attn_t<128, true>(a, st) : launch_attn_t<128, false>(a, st);
-        case 256: return cap ? launch_attn_t<256, true>(a, st) : launch_attn_t<256, false>(a, st);
+        case 64: return cap ? launch_attn_t<64, true, false>(a, st) : launch_attn_t<64, false, false>(a, st);
+        case 128: return cap ? launch_attn_t<128, true, false>(a, st) : launch_attn_t<128, false, false>(a, st);
+        case 256: return cap ? launch_attn_t<256, true, false>(a, st) : launch_attn_t<256, false, false>(a, st);
     }
     return fail(FOCUS_ERR_UNSUPPORTED, "D (%d) must be 64, 128 or 256", a.s.D);
 }

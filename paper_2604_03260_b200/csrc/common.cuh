@@ -45,7 +45,9 @@ int launch_assign(const focus_shape* s, const focus_tensor& x, int H, const floa
                   unsigned long long* near_ties, float eps, cudaStream_t st);
 int launch_assign_hidden(const focus_shape* s, const void* h, int64_t sb, int64_t sn, int d, int dg, const float* Wg,
                          const float* C, const float* bias, float* folded, uint32_t* mq, uint32_t* mk,
-                         unsigned long long* near_ties, float eps, cudaStream_t st);
+                         unsigned long long* near_ties, float eps, float* scores, cudaStream_t st);
+size_t sinkhorn_workspace_bytes(const focus_shape* s, int iters);
+int launch_sinkhorn(const focus_shape* s, const float* S, float tau, int iters, void* ws, float* out, cudaStream_t st);
 size_t decode_workspace_bytes(const focus_shape* s);
 int launch_decode(const focus_shape* s, const focus_tensor& q, const focus_tensor& k, const focus_tensor& v,
                   const uint32_t* mq_new, const uint32_t* mk, const focus_tensor& o, float* lse, float* part, float scale,
@@ -68,6 +70,9 @@ struct AttnArgs {
     float* lse;
     int32_t* dev_status;
     float scale;              // resolved logit scale
+    const float* gate_g = nullptr;   // training-time soft gate: assignments [batch, n, gate_ld]; nullptr = no gate
+    int gate_ld = 0;
+    float gate_lambda = 0.f;
 };
 int launch_attn_simple(const AttnArgs& a, cudaStream_t st);
 int launch_attn_sm100(const AttnArgs& a, cudaStream_t st);
