@@ -28,6 +28,8 @@
 //                   go straight to the rows' original positions
 // Items are laid out KV head by KV head (class-sorted: most key tiles first inside a group) and
 // dealt to the CTAs in alternating direction round by round.
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 #include "tma_host.cuh"
@@ -179,15 +181,17 @@ struct TileWalk {
     }
 };
 
-template <int D>
+template <int D, bool GATE = false>
 struct AttnCfg {
     static constexpr int NQ = (D == 256) ? 1 : 2;            // 128-row query tiles per item
     static constexpr int SUBT = D / 64;
     static constexpr uint32_t SUB_BYTES = 128 * 64 * 2;
     static constexpr uint32_t TILE_BYTES = SUB_BYTES * SUBT;
     // The K/V ring: a stage holds a whole 128-key tile of K or of V.  At D = 256 only two stages fit next to Q.
-    static constexpr int NSTAGE = (D == 256) ? 2 : ((D == 128) ? 5 : 8);
-    static constexpr uint32_t SMEM_BYTES = 1024 + NQ * TILE_BYTES + NSTAGE * TILE_BYTES;
+    static constexpr int NSTAGE = (D == 256) ? 2 : ((D == 128) ? (GATE ? 4 : 5) : 8);
+    // soft gate: per softmax warpgroup two buffers of 128 key assignments, 8 floats each (after the ring)
+    static constexpr uint32_t GATE_BUF_BYTES = 128 * 32;
+    static constexpr uint32_t SMEM_BYTES = 1024 + NQ * TILE_BYTES + NSTAGE * TILE_BYTES + (GATE ? 4 * GATE_BUF_BYTES : 0);
     // Ring order of the tiles.  With one query tile the S of the next key tile is issued before the current P V, so
     // K(next) travels ahead of V(current); with two query tiles V(current) is consumed and released first.
     static constexpr bool K_AHEAD = NQ == 1;
@@ -204,6 +208,7 @@ struct SharedCtl {
     uint64_t s_full[2], p_full[2], o_full[2];
     uint64_t pv_done;
     uint64_t xchg[4];                 // split rows, per 32-row quadrant: both column halves have published a per-row value
+    uint64_t gbar[2];                 // soft gate, per softmax warpgroup: the key assignments of the tile are in shared memory
     uint64_t kv_full[8], kv_empty[8];
     uint32_t tmem_base;
     int abort_flag;
@@ -350,10 +355,10 @@ __device__ __forceinline__ void build_tile_mask_sorted(TileMask& tm, int w, cons
 }
 
 template <int D, bool SOFTCAP, bool GATE>
-__global__ void __launch_bounds__(AttnCfg<D>::THREADS, 1)
+__global__ void __launch_bounds__(AttnCfg<D, GATE>::THREADS, 1)
 focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
-    using C = AttnCfg<D>;
+    using C = AttnCfg<D, GATE>;
     constexpr int NQ = C::NQ;
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) SharedCtl ctl;
@@ -363,6 +368,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sq = base;                                 // NQ query tiles
     const uint32_t skv = base + NQ * C::TILE_BYTES;            // ring of K / V tiles
+    unsigned char* const gate_sm = smem_raw + (base - smem_u32(smem_raw)) + NQ * C::TILE_BYTES + C::NSTAGE * C::TILE_BYTES;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (p.sorted && __ldg(p.counters + 4) != 0ull) {      // more mask values than the sorted layout holds: refuse
@@ -376,6 +382,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         mbar_init(smem_u32(&ctl.q_empty), 1);
         mbar_init(smem_u32(&ctl.pv_done), 1);
         for (int qd = 0; qd < 4; ++qd) mbar_init(smem_u32(&ctl.xchg[qd]), 2);
+        for (int g = 0; g < 2; ++g) mbar_init(smem_u32(&ctl.gbar[g]), 4);
         for (int x = 0; x < 2; ++x) {
             mbar_init(smem_u32(&ctl.s_full[x]), 1);
             mbar_init(smem_u32(&ctl.p_full[x]), 128 * C::NSPLIT);
@@ -611,6 +618,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const float sl2 = SOFTCAP ? p.softcap * LOG2E : p.scale * LOG2E;
         const float cap_in = SOFTCAP ? p.scale / p.softcap : 0.f;
         uint32_t ns = 0;                                     // S tiles consumed by this warpgroup
+        uint32_t ng = 0;                                     // soft gate: tiles whose key assignments this warpgroup has staged
         int it = 0;
         bool ok = true;
         Item t;
@@ -660,6 +668,33 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 } else {
                     build_tile_mask(tm, p, a, kb, i, mi, aq, f_x, hk);
                 }
+                // ---- soft gate (Eq. 2): the score of a distant pair (i - j > w) is multiplied by sigmoid(lambda g_i . g_j).
+                // The warpgroup stages the key assignments of its columns in shared memory before S is needed; every
+                // thread then reads them with broadcast 16-byte loads, column by column.
+                const unsigned char* gb = nullptr;
+                bool gated = false;
+                const long long gj0 = (long long)kb * 128 + half * NC;    // first column of this thread's part of the tile
+                const long long ifar = i - p.w;                           // columns j < ifar are distant for this row
+                if constexpr (GATE) {
+                    // the same decision in all four warps of the warpgroup: does the tile hold a distant pair at all
+                    const bool tile_gated = !tm.all_masked && ((long long)a * 128 + 127 - p.w > gj0);
+                    if (tile_gated) {
+                        unsigned char* gw = gate_sm + (wg * 2 + (ng & 1)) * C::GATE_BUF_BYTES;
+                        const int col = (warp & 3) * 32 + lane;
+                        if (col < NC) {
+                            const long long j = gj0 + col;
+                            const float4* gp = reinterpret_cast<const float4*>(p.gate_g + ((size_t)bb * p.n + (size_t)(j < p.n ? j : p.n - 1)) * p.gate_ld);
+                            reinterpret_cast<float4*>(gw + col * 32)[0] = __ldg(gp);
+                            reinterpret_cast<float4*>(gw + col * 32)[1] = p.gate_ld == 8 ? __ldg(gp + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&ctl.gbar[wg]));
+                        if (!ctl_wait(&ctl.gbar[wg], ng & 1, &ctl)) { report_timeout(p, &ctl, 37, (int)item); ok = false; break; }
+                        ++ng;
+                        gb = gw;
+                        gated = __any_sync(0xffffffffu, valid && ifar > gj0);
+                    }
+                }
                 // ---- wait for S
                 const int buf = NQ == 2 ? x : (int)(ns & 1);
                 const uint32_t par = NQ == 2 ? (ns & 1) : ((ns >> 1) & 1);
@@ -674,34 +709,34 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 } else {
                     uint32_t sr[NC];
 #pragma unroll
-                    for (int c = 0; c < NC / 32; ++c) tmem_ld32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[c * 32]));
+                    for (int c = 0; c < NC / 32; ++c) {
+                        tmem_ld32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[c * 32]));
+                        if constexpr (GATE) {       // chunk by chunk: 32 scores, then their factors
+                            tmem_wait_ld();
+                            if (gated) {
+                                const bool wide = p.gate_ld == 8;
+#pragma unroll
+                                for (int e = 0; e < 32; ++e) {
+                                    const float4* kp = reinterpret_cast<const float4*>(gb + (c * 32 + e) * 32);
+                                    const float4 k0 = kp[0];
+                                    float2 acc = __fmul2_rn(make_float2(gi[0], gi[1]), make_float2(k0.x, k0.y));
+                                    acc = __ffma2_rn(make_float2(gi[2], gi[3]), make_float2(k0.z, k0.w), acc);
+                                    if (wide) {
+                                        const float4 k1 = kp[1];
+                                        acc = __ffma2_rn(make_float2(gi[4], gi[5]), make_float2(k1.x, k1.y), acc);
+                                        acc = __ffma2_rn(make_float2(gi[6], gi[7]), make_float2(k1.z, k1.w), acc);
+                                    }
+                                    const float gate = fmaf(tanh_approx(acc.x + acc.y), 0.5f, 0.5f);
+                                    const float sv = __uint_as_float(sr[c * 32 + e]);
+                                    sr[c * 32 + e] = __float_as_uint(gj0 + c * 32 + e < ifar ? sv * gate : sv);
+                                }
+                            }
+                        }
+                    }
                     tmem_wait_ld();
                     if (SOFTCAP) {
 #pragma unroll
                         for (int c = 0; c < NC; ++c) sr[c] = __float_as_uint(tanh_approx(__uint_as_float(sr[c]) * cap_in));
-                    }
-                    if constexpr (GATE) {
-                        // Eq. 2: the score of a distant pair (i - j > w) is multiplied by sigmoid(lambda g_i . g_j).
-                        // The key assignments are read with warp-uniform addresses (one L1 line serves the warp).
-                        const long long j0 = (long long)kb * 128 + half * NC;
-                        const long long ifar = i - p.w;                   // columns j < ifar are distant for this row
-                        if (__any_sync(0xffffffffu, valid && ifar > j0)) {
-                            const float* gk = p.gate_g + (size_t)bb * p.n * p.gate_ld;
-                            const bool wide = p.gate_ld == 8;
-#pragma unroll
-                            for (int c = 0; c < NC; ++c) {
-                                const long long j = j0 + c;
-                                const float4* gp = reinterpret_cast<const float4*>(gk + (size_t)(j < p.n ? j : p.n - 1) * p.gate_ld);
-                                const float4 a0 = __ldg(gp);
-                                float aff = fmaf(gi[0], a0.x, fmaf(gi[1], a0.y, fmaf(gi[2], a0.z, gi[3] * a0.w)));
-                                if (wide) {
-                                    const float4 a1 = __ldg(gp + 1);
-                                    aff += fmaf(gi[4], a1.x, fmaf(gi[5], a1.y, fmaf(gi[6], a1.z, gi[7] * a1.w)));
-                                }
-                                const float gate = fmaf(tanh_approx(aff), 0.5f, 0.5f);
-                                if (j < ifar) sr[c] = __float_as_uint(__uint_as_float(sr[c]) * gate);
-                            }
-                        }
                     }
                     if (tm.masked) {
 #pragma unroll
@@ -838,7 +873,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
 template <int D, bool SOFTCAP, bool GATE>
 static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
-    using C = AttnCfg<D>;
+    using C = AttnCfg<D, GATE>;
     CUtensorMap tq, tk, tv;
     int rc;
     const bool sorted = a.ws && a.L.layout == FOCUS_LAYOUT_CLASS_SORTED;
