@@ -715,20 +715,34 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             tmem_wait_ld();
                             if (gated) {
                                 const bool wide = p.gate_ld == 8;
+                                const int nfar = (int)(ifar - gj0 < 0 ? 0 : (ifar - gj0 > NC ? NC : ifar - gj0));   // columns < nfar are distant
 #pragma unroll
-                                for (int e = 0; e < 32; ++e) {
-                                    const float4* kp = reinterpret_cast<const float4*>(gb + (c * 32 + e) * 32);
-                                    const float4 k0 = kp[0];
-                                    float2 acc = __fmul2_rn(make_float2(gi[0], gi[1]), make_float2(k0.x, k0.y));
-                                    acc = __ffma2_rn(make_float2(gi[2], gi[3]), make_float2(k0.z, k0.w), acc);
-                                    if (wide) {
-                                        const float4 k1 = kp[1];
-                                        acc = __ffma2_rn(make_float2(gi[4], gi[5]), make_float2(k1.x, k1.y), acc);
-                                        acc = __ffma2_rn(make_float2(gi[6], gi[7]), make_float2(k1.z, k1.w), acc);
+                                for (int e0 = 0; e0 < 32; e0 += 4) {        // four columns in flight
+                                    float4 k0[4], k1[4];
+#pragma unroll
+                                    for (int u = 0; u < 4; ++u) {
+                                        const float4* kp = reinterpret_cast<const float4*>(gb + (c * 32 + e0 + u) * 32);
+                                        k0[u] = kp[0];
+                                        k1[u] = wide ? kp[1] : make_float4(0.f, 0.f, 0.f, 0.f);
                                     }
-                                    const float gate = fmaf(tanh_approx(acc.x + acc.y), 0.5f, 0.5f);
-                                    const float sv = __uint_as_float(sr[c * 32 + e]);
-                                    sr[c * 32 + e] = __float_as_uint(gj0 + c * 32 + e < ifar ? sv * gate : sv);
+                                    float arg[4];
+#pragma unroll
+                                    for (int u = 0; u < 4; ++u) {
+                                        float2 acc = __fmul2_rn(make_float2(gi[0], gi[1]), make_float2(k0[u].x, k0[u].y));
+                                        acc = __ffma2_rn(make_float2(gi[2], gi[3]), make_float2(k0[u].z, k0[u].w), acc);
+                                        if (wide) {
+                                            float2 acb = __fmul2_rn(make_float2(gi[4], gi[5]), make_float2(k1[u].x, k1[u].y));
+                                            acb = __ffma2_rn(make_float2(gi[6], gi[7]), make_float2(k1[u].z, k1[u].w), acb);
+                                            acc = __fadd2_rn(acc, acb);
+                                        }
+                                        arg[u] = acc.x + acc.y;
+                                    }
+#pragma unroll
+                                    for (int u = 0; u < 4; ++u) {
+                                        const float gate = fmaf(tanh_approx(arg[u]), 0.5f, 0.5f);
+                                        const float sv = __uint_as_float(sr[c * 32 + e0 + u]);
+                                        sr[c * 32 + e0 + u] = __float_as_uint(c * 32 + e0 + u < nfar ? sv * gate : sv);
+                                    }
                                 }
                             }
                         }
