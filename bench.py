@@ -34,8 +34,8 @@ UNIT = "TFLOP/s"
 
 # DRAM bytes per launch of the attention kernel (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture per
 # entry, see profiles/), keyed by (workload name, layout); only valid for the kernel sources with this digest.
-ATTN_TRAFFIC = {("M-llama3-8b-128k", 1): 5.68e9}
-ATTN_TRAFFIC_SOURCES = "3b72e6b4b40c7aff"
+ATTN_TRAFFIC = {("M-llama3-8b-128k", 1): 5.87e9}
+ATTN_TRAFFIC_SOURCES = "d391e64345be6987"
 
 
 def attn_traffic(name, layout):
@@ -363,6 +363,24 @@ def main():
         extra["focus_assign_hidden"] = dict(bound="hbm", ms=ms, achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s",
                                             frac=gbs / peaks["hbm_gbs"],
                                             note=f"hidden states [n, {d_model}] bf16, d_g = {d_g}; bytes = 2 d_model per token + the mask rows written")
+        # training-time forward (Sec. 2, Eq. 1 with Sinkhorn normalisation and the Eq. 2 soft gate): scores and Sinkhorn
+        # on the same hidden states, then the gated forward over every causal pair of this workload
+        ld = fb.focus_soft_ld(wl.K)
+        soft = torch.empty((1, wl.n, ld), dtype=torch.float32, device="cuda")
+        ws_sk = torch.empty(fb.focus_sinkhorn_workspace_bytes(shape, 10), dtype=torch.uint8, device="cuda")
+        ms_sc = timed_alone(lambda: fb.focus_router_scores(shape, hid, Wg, Cg, folded, soft))
+        ms_sk = timed_alone(lambda: fb.focus_sinkhorn(shape, soft, 0.1, 10, ws_sk, soft))
+        tr = dict(router_scores_ms=ms_sc, sinkhorn_ms=ms_sk,
+                  note="tau = 0.1, 10 Sinkhorn iterations (12 small launches on an L2-resident score matrix), lambda = 10")
+        if wl.K <= 8 and wl.softcap == 0:
+            O_g, lse_g = torch.empty_like(Q), torch.empty_like(lse)
+            ms_g = timed_alone(lambda: fb.focus_gate_attn_fwd(shape, Q, K, V, soft, 10.0, O_g, lse_g, status), reps=2)
+            del O_g, lse_g
+            gtf = dense_flop / (ms_g * 1e-3) / 1e12
+            tr.update(gate_attn_ms=ms_g, gate_attn_tflops=gtf, bound="alu",
+                      gate_note="every causal pair; 4 D flop per pair on the tensor cores, limited by the per-pair gate "
+                                "(K-term dot product, tanh, two multiplies) on the softmax warps")
+        extra["focus_training_fwd"] = tr
         del hid, flush
 
     # whole-job work: replicas of the workload (weak) or the one workload split by heads (strong)
