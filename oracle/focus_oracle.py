@@ -39,7 +39,7 @@ Passages of the paper each function follows:
 * ``gated_attn``        Sec. 2 "Gated attention" (Eq. 2), the training-time forward over all causal pairs: the
                         score of a distant pair is multiplied by sigmoid(lambda g_i . g_j), a pair inside the
                         window keeps its score.  The equation is followed as printed, so the gate of two
-                        orthogonal assignments is sigmoid(0) = 1/2 (the prose around it says "towards zero").
+                        orthogonal assignments is sigmoid(0) = 1/2 (the prose around it speaks of zero).
 
 Parity status: every function above is pinned by the CPU tests.  "parity unpinned": the paper's
 perplexity and benchmark numbers (datasets and trained weights are not available).
