@@ -187,11 +187,16 @@ struct AttnCfg {
     static constexpr int SUBT = D / 64;
     static constexpr uint32_t SUB_BYTES = 128 * 64 * 2;
     static constexpr uint32_t TILE_BYTES = SUB_BYTES * SUBT;
-    // The K/V ring: a stage holds a whole 128-key tile of K or of V.  At D = 256 only two stages fit next to Q.
-    static constexpr int NSTAGE = (D == 256) ? 2 : ((D == 128) ? (GATE ? 4 : 5) : 8);
+    // The K/V ring.  Up to D = 128 a stage holds a whole 128-key tile of K or of V.  At D = 256 only two such stages
+    // would fit next to Q, so a tile travels as two half stages cut along the contraction dimension of its MMA (the
+    // full-width MMA shapes stay): a K half is all 128 keys x 128 of the 256 head dimensions, a V half is 64 keys x
+    // all 256 dimensions.  Five half stages fit, and a half goes back to the producer as soon as its own MMAs are done.
+    static constexpr int PARTS = (D == 256) ? 2 : 1;         // ring stages per tile
+    static constexpr uint32_t STAGE_BYTES = TILE_BYTES / PARTS;
+    static constexpr int NSTAGE = (D == 256) ? (GATE ? 4 : 5) : ((D == 128) ? (GATE ? 4 : 5) : 8);
     // soft gate: per softmax warpgroup two buffers of 128 key assignments, 8 floats each (after the ring)
     static constexpr uint32_t GATE_BUF_BYTES = 128 * 32;
-    static constexpr uint32_t SMEM_BYTES = 1024 + NQ * TILE_BYTES + NSTAGE * TILE_BYTES + (GATE ? 4 * GATE_BUF_BYTES : 0);
+    static constexpr uint32_t SMEM_BYTES = 1024 + NQ * TILE_BYTES + NSTAGE * STAGE_BYTES + (GATE ? 4 * GATE_BUF_BYTES : 0);
     // Ring order of the tiles.  With one query tile the S of the next key tile is issued before the current P V, so
     // K(next) travels ahead of V(current); with two query tiles V(current) is consumed and released first.
     static constexpr bool K_AHEAD = NQ == 1;
@@ -363,12 +368,13 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) SharedCtl ctl;
     // split rows: [parity][column half][row] row maxima, at the end row sums (the other instantiations have no room to spare)
-    __shared__ float xval_s[C::NSPLIT == 2 ? 2 * 2 * 128 : 1];
-    auto xval = [&](int par, int hf, int row) -> float& { return xval_s[C::NSPLIT == 2 ? (par * 2 + hf) * 128 + row : 0]; };
+    // (bf16: a rounded row maximum serves as well as the exact one as long as both threads use the same value)
+    __shared__ __nv_bfloat16 xval_s[C::NSPLIT == 2 ? 2 * 2 * 128 : 1];
+    auto xval = [&](int par, int hf, int row) -> __nv_bfloat16& { return xval_s[C::NSPLIT == 2 ? (par * 2 + hf) * 128 + row : 0]; };
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sq = base;                                 // NQ query tiles
     const uint32_t skv = base + NQ * C::TILE_BYTES;            // ring of K / V tiles
-    unsigned char* const gate_sm = smem_raw + (base - smem_u32(smem_raw)) + NQ * C::TILE_BYTES + C::NSTAGE * C::TILE_BYTES;
+    unsigned char* const gate_sm = smem_raw + (base - smem_u32(smem_raw)) + NQ * C::TILE_BYTES + C::NSTAGE * C::STAGE_BYTES;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (p.sorted && __ldg(p.counters + 4) != 0ull) {      // more mask values than the sorted layout holds: refuse
@@ -429,21 +435,29 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     for (int c = 0; c < C::SUBT; ++c)
                         tma_load_4d(sq + x * C::TILE_BYTES + c * C::SUB_BYTES, &tm_q, smem_u32(&ctl.q_full), c * 64,
                                     (A * NQ + x) * 128, qh, qb);
-                // one K or V tile into the next stage of the ring
+                // one K or V tile into the next stage(s) of the ring
                 auto load_tile = [&](bool is_v, int tile) {
-                    const int slot = (int)(nload % C::NSTAGE);
-                    const long long use = nload / C::NSTAGE;
-                    if (use > 0 && !ctl_wait(&ctl.kv_empty[slot], (uint32_t)((use - 1) & 1), &ctl)) {
-                        report_timeout(p, &ctl, 11, (int)item);
-                        ok = false;
-                        return;
+                    for (int part = 0; part < C::PARTS; ++part) {
+                        const int slot = (int)(nload % C::NSTAGE);
+                        const long long use = nload / C::NSTAGE;
+                        if (use > 0 && !ctl_wait(&ctl.kv_empty[slot], (uint32_t)((use - 1) & 1), &ctl)) {
+                            report_timeout(p, &ctl, 11, (int)item);
+                            ok = false;
+                            return;
+                        }
+                        const uint32_t bar = smem_u32(&ctl.kv_full[slot]);
+                        const uint32_t dst = skv + slot * C::STAGE_BYTES;
+                        mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
+                        if (is_v) {     // 128 / PARTS keys x all dimensions: one box of 64 columns x 128 / PARTS rows per sub-tile
+                            for (int c = 0; c < C::SUBT; ++c)
+                                tma_load_4d(dst + c * (C::SUB_BYTES / C::PARTS), &tm_v, bar, c * 64, tile * 128 + part * (128 / C::PARTS),
+                                            kh, qb);
+                        } else {        // all keys x D / PARTS dimensions
+                            for (int c = 0; c < C::SUBT / C::PARTS; ++c)
+                                tma_load_4d(dst + c * C::SUB_BYTES, &tm_k, bar, (part * (C::SUBT / C::PARTS) + c) * 64, tile * 128, kh, qb);
+                        }
+                        ++nload;
                     }
-                    const uint32_t bar = smem_u32(&ctl.kv_full[slot]);
-                    mbar_arrive_expect_tx(bar, C::TILE_BYTES);
-                    for (int c = 0; c < C::SUBT; ++c)
-                        tma_load_4d(skv + slot * C::TILE_BYTES + c * C::SUB_BYTES, is_v ? &tm_v : &tm_k, bar, c * 64, tile * 128,
-                                    kh, qb);
-                    ++nload;
                 };
                 if constexpr (C::K_AHEAD) {
                     // load order K(0), then per tile K(next), V(current): the K of the next tile is needed first (its
@@ -480,7 +494,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             bool ok = true;
             const uint64_t qdesc0 = smem_desc_sw128(sq, 16, 1024);
             const uint64_t kvdesc0 = smem_desc_sw128(skv, 16, 1024);             // K tiles: K-major
-            const uint64_t vdesc0 = smem_desc_sw128(skv, C::SUB_BYTES, 1024);     // V tiles: MN-major
+            const uint64_t vdesc0 = smem_desc_sw128(skv, C::SUB_BYTES / C::PARTS, 1024);     // V tiles: MN-major, 64-column chunks
             // S[buf] = Q_x K^T
             auto issue_s = [&](int x, int buf, int kslot) {
                 if (elect_one()) {
@@ -489,7 +503,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks) {
                         const uint64_t off = (uint64_t)(((ks / 4) * C::SUB_BYTES + (ks % 4) * 32) >> 4);
-                        umma_ss(d, ad + off, kvdesc0 + (uint64_t)((kslot * C::TILE_BYTES) >> 4) + off, IDESC_S, ks > 0);
+                        umma_ss(d, ad + off, kvdesc0 + (uint64_t)((kslot * C::STAGE_BYTES) >> 4) + off, IDESC_S, ks > 0);
                     }
                 }
             };
@@ -498,7 +512,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (elect_one()) {
                     const uint32_t d = tmem + (x ? C::COL_O1 : C::COL_O0);
                     const uint32_t a = tmem + (buf ? C::COL_S1 : C::COL_S0);
-                    const uint64_t bd = vdesc0 + (uint64_t)((vslot * C::TILE_BYTES) >> 4);
+                    const uint64_t bd = vdesc0 + (uint64_t)((vslot * C::STAGE_BYTES) >> 4);
                     // split rows: the P of column half h sits at columns 64 h .. 64 h + 31
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)
@@ -521,6 +535,49 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 ++nuse;
                 return true;
             };
+            // One query tile: S[buf] = Q K^T and O (+)= P[buf] V stage by stage -- wait for the stage, issue the MMAs that
+            // read it, hand it back.  The stages are taken in the ring's order: K(next) before V(current).
+            auto s_tile = [&](int buf, int where, int item) -> bool {
+                constexpr int KS = D / 16 / C::PARTS;            // k-steps per stage
+                const uint32_t d = tmem + (buf ? C::COL_S1 : C::COL_S0);
+                for (int part = 0; part < C::PARTS; ++part) {
+                    int slot;
+                    if (!wait_kv(slot, where, item)) return false;
+                    tc_fence_after();
+                    if (elect_one()) {
+#pragma unroll
+                        for (int k2 = 0; k2 < KS; ++k2) {
+                            const int ks = part * KS + k2;
+                            const uint64_t qoff = (uint64_t)(((ks / 4) * C::SUB_BYTES + (ks % 4) * 32) >> 4);
+                            const uint64_t koff = (uint64_t)((slot * C::STAGE_BYTES + (k2 / 4) * C::SUB_BYTES + (k2 % 4) * 32) >> 4);
+                            umma_ss(d, qdesc0 + qoff, kvdesc0 + koff, IDESC_S, ks > 0);
+                        }
+                    }
+                    release_tile(slot);
+                }
+                commit(&ctl.s_full[buf]);
+                return true;
+            };
+            auto o_tile = [&](int buf, bool first, int where, int item) -> bool {
+                constexpr int KS = 8 / C::PARTS;
+                const uint32_t d = tmem + C::COL_O0;
+                const uint32_t a = tmem + (buf ? C::COL_S1 : C::COL_S0);
+                for (int part = 0; part < C::PARTS; ++part) {
+                    int slot;
+                    if (!wait_kv(slot, where, item)) return false;
+                    tc_fence_after();
+                    if (elect_one()) {
+#pragma unroll
+                        for (int k2 = 0; k2 < KS; ++k2) {
+                            const int ks = part * KS + k2;
+                            umma_ts(d, a + (C::NSPLIT == 2 ? (ks / 4) * 64 + (ks % 4) * 8 : ks * 8),
+                                    vdesc0 + (uint64_t)((slot * C::STAGE_BYTES + k2 * 2048) >> 4), IDESC_O, (!first) || ks > 0);
+                        }
+                    }
+                    release_tile(slot);
+                }
+                return true;
+            };
             Item t;
             for (int round = 0; ok && item_of(p, round, t); ++round) {
                 const int A = t.A, hq = t.hq;
@@ -530,35 +587,29 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 int cur = walk.next();
                 if (cur < 0) continue;
                 if (!ctl_wait(&ctl.q_full, it & 1, &ctl)) { report_timeout(p, &ctl, 20, (int)item); break; }
-                int slot;
-                if (!wait_kv(slot, 21, (int)item)) break;
-                tc_fence_after();
                 if constexpr (NQ == 2) {
+                    int slot;
+                    if (!wait_kv(slot, 21, (int)item)) break;
+                    tc_fence_after();
                     issue_s(0, 0, slot); commit(&ctl.s_full[0]);
                     issue_s(1, 1, slot); commit(&ctl.s_full[1]);
                     release_tile(slot);
                 } else {
-                    issue_s(0, gs & 1, slot);
-                    commit(&ctl.s_full[gs & 1]);
-                    release_tile(slot);
+                    if (!s_tile(gs & 1, 21, (int)item)) break;
                     ++gs;
                 }
                 bool first = true;
                 while (cur >= 0) {
                     const int nxt = walk.next();
-                    int vslot, kslot = 0;
-                    // the ring order of K(next) and V(current) is the producer's
-                    if constexpr (!C::K_AHEAD) {
+                    int vslot = 0, kslot = 0;
+                    if constexpr (NQ == 2) {
+                        // the ring carries V(current) ahead of K(next) here (see the producer)
                         if (!wait_kv(vslot, 22, (int)item)) { ok = false; break; }
+                        if (nxt >= 0) {
+                            if (!wait_kv(kslot, 23, (int)item)) { ok = false; break; }
+                        }
                     }
-                    if (nxt >= 0) {
-                        if (!wait_kv(kslot, 23, (int)item)) { ok = false; break; }
-                    } else {
-                        commit(&ctl.q_empty);     // every S of this item has been issued
-                    }
-                    if constexpr (C::K_AHEAD) {
-                        if (!wait_kv(vslot, 22, (int)item)) { ok = false; break; }
-                    }
+                    if (nxt < 0) commit(&ctl.q_empty);     // every S of this item has been issued
                     if constexpr (NQ == 2) {
                         // query tile 0
                         if (!ctl_wait(&ctl.p_full[0], np[0] & 1, &ctl)) { report_timeout(p, &ctl, 24, (int)item); ok = false; break; }
@@ -582,17 +633,14 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     } else {
                         // S of the next tile goes to the other buffer before this tile's PV is issued
                         if (nxt >= 0) {
-                            issue_s(0, gs & 1, kslot);
-                            commit(&ctl.s_full[gs & 1]);
-                            release_tile(kslot);
+                            if (!s_tile(gs & 1, 23, (int)item)) { ok = false; break; }
                             ++gs;
                         }
                         const int buf = gp & 1;
                         if (!ctl_wait(&ctl.p_full[buf], (gp >> 1) & 1, &ctl)) { report_timeout(p, &ctl, 26, (int)item); ok = false; break; }
                         ++gp;
                         tc_fence_after();
-                        issue_o(0, buf, vslot, first);
-                        release_tile(vslot);
+                        if (!o_tile(buf, first, 22, (int)item)) { ok = false; break; }
                         commit(&ctl.pv_done);
                         if (nxt < 0) commit(&ctl.o_full[0]);
                     }
@@ -770,11 +818,12 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     if constexpr (NSPLIT == 2) {
                         // the two threads of a row exchange the maxima of their halves and then take the same decisions
                         const int par = (int)(nx & 1);
-                        xval(par, half, row_in_tile) = mraw;
+                        const __nv_bfloat16 mine = __float2bfloat16_rn(mraw);
+                        xval(par, half, row_in_tile) = mine;
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&ctl.xchg[warp & 3]));
                         if (!ctl_wait(&ctl.xchg[warp & 3], (uint32_t)par, &ctl)) { report_timeout(p, &ctl, 36, (int)item); ok = false; }
-                        mraw = fmaxf(mraw, xval(par, half ^ 1, row_in_tile));
+                        mraw = fmaxf(__bfloat162float(mine), __bfloat162float(xval(par, half ^ 1, row_in_tile)));
                         ++nx;
                     }
                     const float mt = mraw * sl2;                     // log2 units (sl2 > 0; -inf stays -inf)
@@ -843,14 +892,22 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             if (!ok) break;
             // ---- epilogue: O / l -> bf16 -> global, lse
             if constexpr (NSPLIT == 2) {
-                // the two halves add their row sums
-                const int par = (int)(nx & 1);
-                xval(par, half, row_in_tile) = l;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl.xchg[warp & 3]));
-                if (!ctl_wait(&ctl.xchg[warp & 3], (uint32_t)par, &ctl)) { report_timeout(p, &ctl, 38, (int)item); break; }
-                l += xval(par, half ^ 1, row_in_tile);
-                ++nx;
+                // the two halves add their row sums: two exchanges, the leading bf16 part of the sum and its remainder
+                float other = 0.f, rest = l;
+                bool xok = true;
+                for (int piece = 0; piece < 2 && xok; ++piece) {
+                    const int par = (int)(nx & 1);
+                    const __nv_bfloat16 mine = __float2bfloat16_rn(rest);
+                    rest -= __bfloat162float(mine);
+                    xval(par, half, row_in_tile) = mine;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl.xchg[warp & 3]));
+                    xok = ctl_wait(&ctl.xchg[warp & 3], (uint32_t)par, &ctl);
+                    other += __bfloat162float(xval(par, half ^ 1, row_in_tile));
+                    ++nx;
+                }
+                if (!xok) { report_timeout(p, &ctl, 38, (int)item); break; }
+                l += other;
             }
             if (!ctl_wait(&ctl.o_full[x], it & 1, &ctl)) { report_timeout(p, &ctl, 40 + x, (int)item); break; }
             tc_fence_after();
@@ -903,11 +960,11 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
         const focus_tensor sv_t{ws + a.L.vs, (int64_t)HK * a.L.nkp * D, (int64_t)a.L.nkp * D, D};
         if ((rc = make_tmap_qkv(&tq, sq_t, 1, HQ, a.L.nqp, D))) return rc;
         if ((rc = make_tmap_qkv(&tk, sk_t, 1, HK, a.L.nkp, D))) return rc;
-        if ((rc = make_tmap_qkv(&tv, sv_t, 1, HK, a.L.nkp, D))) return rc;
+        if ((rc = make_tmap_qkv(&tv, sv_t, 1, HK, a.L.nkp, D, 128 / C::PARTS))) return rc;
     } else {
         if ((rc = make_tmap_qkv(&tq, a.q, a.s.batch, a.s.Hq, a.s.n, D))) return rc;
         if ((rc = make_tmap_qkv(&tk, a.k, a.s.batch, a.s.Hkv, a.s.n, D))) return rc;
-        if ((rc = make_tmap_qkv(&tv, a.v, a.s.batch, a.s.Hkv, a.s.n, D))) return rc;
+        if ((rc = make_tmap_qkv(&tv, a.v, a.s.batch, a.s.Hkv, a.s.n, D, 128 / C::PARTS))) return rc;
     }
     AttnParams p;
     p.B = a.s.batch; p.Hq = a.s.Hq; p.Hkv = a.s.Hkv; p.G = a.s.Hq / a.s.Hkv; p.n = a.s.n; p.w = a.s.window; p.K = a.s.K;

@@ -12,7 +12,7 @@ namespace focus {
 int make_tmap_bf16_4d(CUtensorMap* out, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t d3,
                       uint64_t s1_bytes, uint64_t s2_bytes, uint64_t s3_bytes, uint32_t box0, uint32_t box1);
 
-// tensor map of a [batch, H, n, D] bf16 focus_tensor with a 64 x 128 (columns x rows) box
-int make_tmap_qkv(CUtensorMap* out, const focus_tensor& t, int batch, int H, int n, int D);
+// tensor map of a [batch, H, n, D] bf16 focus_tensor with a 64 x rows (columns x rows) box
+int make_tmap_qkv(CUtensorMap* out, const focus_tensor& t, int batch, int H, int n, int D, int rows = 128);
 
 }  // namespace focus
