@@ -110,3 +110,29 @@ def test_auto_layout_is_resolved_from_the_shape():
     assert fb.focus_tiles_workspace_bytes(s, fb.FOCUS_LAYOUT_AUTO) == fb.focus_tiles_workspace_bytes(s, 1)
     L = fb.focus_tiles_layout()
     assert fb.lib().focus_tiles_layout_of(ctypes.byref(s), 3, ctypes.byref(L)) == -1
+
+
+def test_training_forward_host_checks():
+    """row length of the soft assignments, Sinkhorn workspace size, and argument checks that precede any launch"""
+    L = fb.lib()
+    assert [fb.focus_soft_ld(K) for K in (1, 4, 5, 8, 9, 16, 17, 32)] == [4, 4, 8, 8, 16, 16, 32, 32]
+    assert fb.focus_soft_ld(0) == 0 and fb.focus_soft_ld(33) == 0
+    s = fb.make_shape(8, 2, 1000, 128, 8, 2, 64, batch=3)
+    w10, w20 = fb.focus_sinkhorn_workspace_bytes(s, 10), fb.focus_sinkhorn_workspace_bytes(s, 20)
+    assert w10 > 0 and w20 > w10 and w10 % 16 == 0
+    assert fb.focus_sinkhorn_workspace_bytes(s, 0) == 0
+    assert fb.focus_sinkhorn_workspace_bytes(fb.make_shape(8, 2, 1000, 128, 8, 2, 64, batch=1), 10) * 3 == w10   # per sequence
+    assert L.focus_sinkhorn(ctypes.byref(s), None, 0.1, 10, 4096, w10, 4096, None) == -1          # scores NULL
+    assert L.focus_sinkhorn(ctypes.byref(s), 4096, 0.0, 10, 4096, w10, 4096, None) == -1           # temperature
+    assert L.focus_sinkhorn(ctypes.byref(s), 4096, 0.1, 0, 4096, w10, 4096, None) == -1            # iterations
+    assert L.focus_sinkhorn(ctypes.byref(s), 4096, 0.1, 10, 4096, 8, 4096, None) == -3             # capacity
+    assert L.focus_sinkhorn(ctypes.byref(s), 4100, 0.1, 10, 4096, w10, 4096, None) == -1           # alignment
+    assert L.focus_router_scores(ctypes.byref(s), 4096, 1000 * 512, 512, 512, 16, 4096, 4096, 4096, None, None) == -1
+    assert L.focus_router_scores(ctypes.byref(s), 4096, 1000 * 512, 512, 510, 16, 4096, 4096, 4096, 4096, None) == -1   # d_model % 8
+    t_ok = fb.focus_tensor(4096, 8 * 1000 * 128, 1000 * 128, 128)
+    assert L.focus_gate_attn_fwd(ctypes.byref(s), t_ok, t_ok, t_ok, None, 5.0, t_ok, 4096, None, None) == -1     # g NULL
+    assert L.focus_gate_attn_fwd(ctypes.byref(s), t_ok, t_ok, t_ok, 4100, 5.0, t_ok, 4096, None, None) == -1     # g alignment
+    capped = fb.make_shape(8, 2, 1000, 128, 8, 2, 64, softcap=30.0)
+    assert L.focus_gate_attn_fwd(ctypes.byref(capped), t_ok, t_ok, t_ok, 4096, 5.0, t_ok, 4096, None, None) == -2   # unsupported
+    many = fb.make_shape(8, 2, 1000, 128, 16, 2, 64)
+    assert L.focus_gate_attn_fwd(ctypes.byref(many), t_ok, t_ok, t_ok, 4096, 5.0, t_ok, 4096, None, None) == -2
