@@ -150,7 +150,8 @@ def run_reference(args, wl):
 def run_sweep(args):
     """--sweep: context-length sweep in the shape of the paper's speedup table (Sec. 3.6 / Table 6): Llama-3-8B-shaped
     layer (32/8 heads, D=128, w=2048), n = 1K ... 1M, K in {4, 8}, top-k in {1, 2}; per point the same kernel in
-    dense-causal mode, the original layout and the class-sorted layout (gathers included), one JSON line each."""
+    dense-causal mode, the original layout and the two class-sorted layouts (gathers, window pass and merge included), one
+    JSON line each."""
     from paper_2604_03260_b200 import binding as fb
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     ev = lambda: torch.cuda.Event(enable_timing=True)
@@ -180,7 +181,7 @@ def run_sweep(args):
             reps = 3 if n <= 262144 else 1
             row = dict(sweep=True, n=n, K=K, topk=topk, window=wl.window, Hq=32, Hkv=8, D=128)
             row["dense_ms"] = timed(lambda: fb.focus_attn_fwd(shape, Q, Kt, V, None, None, None, 0, O, lse, status), reps)
-            for layout, name in ((0, "original"), (1, "sorted")):
+            for layout, name in ((0, "original"), (1, "sorted"), (3, "sorted_local")):
                 ws = fb.alloc_workspace(shape, layout)
                 row[f"tiles_{name}_ms"] = timed(lambda: fb.focus_build_tiles(shape, mq, mk, layout, ws), reps)
                 row[f"{name}_ms"] = timed(lambda: fb.focus_attn_fwd(shape, Q, Kt, V, mq, mk, ws, layout, O, lse, status), reps)
@@ -191,7 +192,9 @@ def run_sweep(args):
                     row["kept_fraction"] = cnt.sum().item() / wl.dense_pairs()
                 del ws
             assert status[0].item() == 0, status.tolist()
-            best = min(row["original_ms"] + row["tiles_original_ms"], row["sorted_ms"] + row["tiles_sorted_ms"])
+            best = min(row["original_ms"] + row["tiles_original_ms"], row["sorted_ms"] + row["tiles_sorted_ms"],
+                       row["sorted_local_ms"] + row["tiles_sorted_local_ms"])
+            row["auto_layout"] = fb.focus_tiles_layout_of(shape, fb.FOCUS_LAYOUT_AUTO).layout
             row["speedup_vs_dense"] = row["dense_ms"] / best
             row["kept_tflops_best"] = 4.0 * wl.D * row["kept_fraction"] * wl.dense_pairs() / (best * 1e-3) / 1e12
             print(json.dumps(row), flush=True)
@@ -206,7 +209,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="focus", choices=["focus", "reference"])
     ap.add_argument("--workload", default="M128k")
-    ap.add_argument("--layout", type=int, default=1, help="0 = original token order, 1 = class-sorted (group-permuted), 2 = chosen by the library from the shape")
+    ap.add_argument("--layout", type=int, default=1, help="0 = original token order, 1 = class-sorted (group-permuted), 2 = chosen by the library from the shape, "
+                                                           "3 = class-sorted for sharing pairs + window pass in token order")
     ap.add_argument("--ref-rows", type=int, default=2048, help="oracle rows per step (reference arm)")
     ap.add_argument("--cpu-rows", type=int, default=24576, help="oracle rows of the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -257,7 +261,8 @@ def main():
     lse = torch.empty((wl.Hq, wl.n), dtype=torch.float32, device="cuda")
     status = torch.zeros(4, dtype=torch.int32, device="cuda")
     # assign x2, build_tiles (4 kernels; class-sorted: + 6 per side + ranges + order), attention (+ 3 gathers)
-    launches_per_step = 2 + 4 + 1 + (14 + 3 if layout == 1 else 0)
+    # layout 3: + fill, second attention launch, merge
+    launches_per_step = 2 + 4 + 1 + (14 + 3 if layout in (1, 3) else 0) + (3 if layout == 3 else 0)
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
     marks = []
@@ -469,7 +474,7 @@ def main():
                         parallelism=("single GPU" if world == 1 else
                                      f"{world} replicas, no collective" if args.scaling == "weak" else
                                      f"KV heads split over {world} ranks, no collective"),
-                        softcap=wl.softcap, layout=["original", "class-sorted"][layout],
+                        softcap=wl.softcap, layout=["original", "class-sorted", None, "class-sorted + window pass"][layout],
                         l2="inputs larger than L2 (Q+K+V+O = %.2f GiB); no flush between steps" %
                            ((2 * Q.numel() + 2 * K.numel()) * 2 / 2**30)),
             clocks=clocks,

@@ -74,12 +74,21 @@ typedef struct {
 
 #define FOCUS_LAYOUT_ORIGINAL 0
 #define FOCUS_LAYOUT_CLASS_SORTED 1
-/* Let the library choose between the two from the shape alone (n, K, topk): the class-sorted layout when the
+/* Let the library choose from the shape alone (n, K, topk, window): a class-sorted layout when the
  * sequence is long enough for its fixed costs (at least 16384 tokens and 2048 per mask class, C(K, topk) classes
  * assumed) and enough distant pairs fall away (at least half of them for uniform memberships, or at least 15 % from
- * 65536 tokens on); the original layout otherwise.  focus_tiles_layout_of reports the choice in `layout`; pass
+ * 65536 tokens on); the original layout otherwise.  Of the two class-sorted layouts FOCUS_LAYOUT_SORTED_LOCAL is taken
+ * when the window of a block of sorted queries, spread over the C(K-topk, topk) classes it shares no group with,
+ * would cost over 1.25 times the key tiles of a window pass in token order, fixed costs included (many classes: K = 8).
+ * focus_tiles_layout_of reports the choice in `layout`; pass
  * the same value to focus_tiles_workspace_bytes, focus_build_tiles and focus_attn_fwd. */
 #define FOCUS_LAYOUT_AUTO 2
+/* Class-sorted layout for the pairs that share a group, plus a second pass in the original token order for the
+ * pairs that are attended only because they lie inside the window (no shared group); the two partial results
+ * cover disjoint sets of pairs and are joined through their logsumexps (paper Appendix C, "Disjoint decomposition"
+ * and "Merge").  With many small classes the sorted order scatters the window of a query block over a wide range
+ * of every other class; the separate pass reads the window once, in token order. */
+#define FOCUS_LAYOUT_SORTED_LOCAL 3
 
 /*
  * Byte offsets of the arrays inside a tiles workspace (a pure function of shape and layout;
@@ -114,6 +123,10 @@ typedef struct {
                                 group, most key tiles first */
     size_t qs, ks, vs;       /* bf16 sorted copies [B*Hq][nqp][D], [B*Hkv][nkp][D] x2, filled by focus_attn_fwd */
     size_t scratch;          /* build-time scratch (hash sets of mask values, chunk histograms, block costs) */
+    /* FOCUS_LAYOUT_SORTED_LOCAL only (0 otherwise): the two partial results, kept in fp32 until they are joined */
+    size_t o_sorted;         /* fp32 [B*Hq][n][D]: class-sorted pass (its logsumexp goes to the caller's lse) */
+    size_t o_local;          /* fp32 [B*Hq][n][D]: window pass */
+    size_t lse_local;        /* fp32 [B*Hq][n] */
 } focus_tiles_layout;
 
 /* Library version (major*10000 + minor*100 + patch). */
@@ -194,7 +207,8 @@ FOCUS_API int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, co
  *   mq, mk      device masks; may be NULL when tiles_ws is NULL
  *   tiles_ws    workspace written by focus_build_tiles for the same shape and masks.  NULL = dense
  *               causal mode (every causal pair attended; masks and layout ignored).
- *   layout      the layout the workspace was built with: FOCUS_LAYOUT_ORIGINAL walks tiles in token
+ *   layout      the layout the workspace was built with (FOCUS_LAYOUT_SORTED_LOCAL: the class-sorted pass over
+ *               sharing pairs, the window pass in token order, then a merge kernel): FOCUS_LAYOUT_ORIGINAL walks tiles in token
  *               order and skips dead far tiles; FOCUS_LAYOUT_CLASS_SORTED gathers Q/K/V into the
  *               class-sorted order kept in the workspace, walks only sharing class pairs plus the
  *               window, and scatters O/lse back to token order.

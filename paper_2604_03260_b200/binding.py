@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libfocus_b200.so")
 FOCUS_LAYOUT_ORIGINAL = 0
 FOCUS_LAYOUT_CLASS_SORTED = 1
 FOCUS_LAYOUT_AUTO = 2
+FOCUS_LAYOUT_SORTED_LOCAL = 3
 FOCUS_MAX_CLASSES = 64
 
 
@@ -39,7 +40,8 @@ class focus_tiles_layout(C.Structure):
                 ("cnt_q", C.c_size_t), ("cnt_k", C.c_size_t),
                 ("seg_q", C.c_size_t), ("seg_k", C.c_size_t), ("perm_q", C.c_size_t), ("perm_k", C.c_size_t),
                 ("qrange", C.c_size_t), ("order", C.c_size_t), ("qs", C.c_size_t), ("ks", C.c_size_t),
-                ("vs", C.c_size_t), ("scratch", C.c_size_t)]
+                ("vs", C.c_size_t), ("scratch", C.c_size_t), ("o_sorted", C.c_size_t), ("o_local", C.c_size_t),
+                ("lse_local", C.c_size_t)]
 
 
 class FocusError(RuntimeError):

@@ -82,7 +82,17 @@ static int choose_layout(const focus_shape* s) {
     const double dropped = binom(s->K - s->topk, s->topk) / classes;      // far pairs without a shared group, uniform memberships
     const double min_n = classes * 2048.0 > 16384.0 ? classes * 2048.0 : 16384.0;
     if ((double)s->n < min_n) return FOCUS_LAYOUT_ORIGINAL;
-    if (dropped >= 0.5 || (s->n >= 65536 && dropped >= 0.15)) return FOCUS_LAYOUT_CLASS_SORTED;
+    if (dropped >= 0.5 || (s->n >= 65536 && dropped >= 0.15)) {
+        // Key tiles a block of 256 sorted queries visits for its window alone: its rows span about 256 * classes
+        // positions, so the window of the block covers (256 * classes + w) / classes keys of every class that shares
+        // no group with it.  The separate window pass in token order reads w + 256 keys once per 256 rows, plus what
+        // a second pass costs per block whatever its length (query load, pipeline fill, fp32 partial results, merge):
+        // about six key tiles' worth, measured.  The pass is taken when it saves a quarter or more.
+        const double apart = binom(s->K - s->topk, s->topk);                 // classes without a shared group
+        const double in_sorted = apart * ((256.0 * classes + s->window) / classes / 128.0 + 1.0);
+        const double in_order = (s->window + 256.0) / 128.0 + 7.0;
+        return in_sorted > 1.25 * in_order ? FOCUS_LAYOUT_SORTED_LOCAL : FOCUS_LAYOUT_CLASS_SORTED;
+    }
     return FOCUS_LAYOUT_ORIGINAL;
 }
 
@@ -91,8 +101,9 @@ static int layout_of(const focus_shape* s, int layout, focus_tiles_layout* L) {
     if (rc) return rc;
     if (!L) return fail(FOCUS_ERR_INVALID_ARG, "out is NULL");
     if (layout == FOCUS_LAYOUT_AUTO) layout = choose_layout(s);
-    if (layout != FOCUS_LAYOUT_ORIGINAL && layout != FOCUS_LAYOUT_CLASS_SORTED)
-        return fail(FOCUS_ERR_INVALID_ARG, "layout must be 0 (original), 1 (class-sorted) or 2 (chosen by the library)");
+    if (layout != FOCUS_LAYOUT_ORIGINAL && layout != FOCUS_LAYOUT_CLASS_SORTED && layout != FOCUS_LAYOUT_SORTED_LOCAL)
+        return fail(FOCUS_ERR_INVALID_ARG,
+                    "layout must be 0 (original), 1 (class-sorted), 2 (chosen by the library) or 3 (class-sorted + window pass)");
     memset(L, 0, sizeof *L);
     const size_t HQ = (size_t)s->batch * s->Hq, HK = (size_t)s->batch * s->Hkv;
     L->layout = layout;
@@ -111,7 +122,7 @@ static int layout_of(const focus_shape* s, int layout, focus_tiles_layout* L) {
     L->live_cnt = take(HQ * L->nqt * 4);
     L->kany = take(HK * (size_t)s->K * L->nkw * 4);
     L->kall = take(HK * (size_t)s->K * L->nkw * 4);
-    if (layout == FOCUS_LAYOUT_CLASS_SORTED) {
+    if (layout == FOCUS_LAYOUT_CLASS_SORTED || layout == FOCUS_LAYOUT_SORTED_LOCAL) {
         L->nqp = sorted_capacity(s->n);
         L->nkp = sorted_capacity(s->n);
         L->ncls_q = take(HQ * 4);
@@ -130,6 +141,11 @@ static int layout_of(const focus_shape* s, int layout, focus_tiles_layout* L) {
         L->ks = take(HK * (size_t)L->nkp * s->D * 2);
         L->vs = take(HK * (size_t)L->nkp * s->D * 2);
         L->scratch = take(sorted_scratch_bytes(s));
+    }
+    if (layout == FOCUS_LAYOUT_SORTED_LOCAL) {
+        L->o_sorted = take(HQ * (size_t)s->n * s->D * 4);
+        L->o_local = take(HQ * (size_t)s->n * s->D * 4);
+        L->lse_local = take(HQ * (size_t)s->n * 4);
     }
     L->total_bytes = off;
     return FOCUS_OK;
@@ -243,7 +259,7 @@ int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, const uint32
     if (ws_bytes < L.total_bytes)
         return fail(FOCUS_ERR_CAPACITY, "workspace has %zu bytes, %zu needed", ws_bytes, L.total_bytes);
     layout = L.layout;                     // FOCUS_LAYOUT_AUTO resolved
-    if (layout == FOCUS_LAYOUT_CLASS_SORTED) {
+    if (layout == FOCUS_LAYOUT_CLASS_SORTED || layout == FOCUS_LAYOUT_SORTED_LOCAL) {
         // masks with exactly topk bits have C(K, topk) values; more than the class table holds is refused here,
         // other mask patterns with too many values are caught on the device (counters[4], then dev_status)
         double classes = 1.0;

@@ -109,6 +109,9 @@ struct AttnParams {
     const float* gate_g;
     int gate_ld;
     float gate_hl;
+    // window pass of the split layout: only the tiles that reach into the window, only pairs WITHOUT a shared group
+    int local_only;
+    float* o32;              // partial passes: O in fp32, rows [B*Hq][n][D], instead of bf16 to `o`
 };
 
 // Enumerates the key tiles a 256-row query block visits, in increasing order.  Every role of the
@@ -145,7 +148,7 @@ struct TileWalk {
             l0 = p.live + ((size_t)hq * p.nqt + a0) * p.nkw;
             if (nq > 1 && a0 + 1 < p.nqt) l1 = l0 + p.nkw;
         }
-        far_phase = f0 > 0;
+        far_phase = f0 > 0 && !p.local_only;
         wd = -1;
         bits = 0;
         b = f0;
@@ -257,7 +260,9 @@ __device__ __forceinline__ void build_tile_mask(TileMask& tm, const AttnParams& 
     const bool need_causal = c0 + 127 > r_first;
     bool need_group = false, need_window = false;
     if (!p.dense && !tm.all_masked) {
-        if (kb < f_x) {
+        if (p.local_only) {
+            need_group = need_window = true;
+        } else if (kb < f_x) {
             need_group = !(aq & __ldg(p.andk + (size_t)hk * p.nkt + kb));
         } else if (r_last - c0 > p.w) {
             need_group = need_window = true;
@@ -284,7 +289,8 @@ __device__ __forceinline__ void build_tile_mask(TileMask& tm, const AttnParams& 
                 keep = sh[q];
                 if (need_window) {
                     const long long lo = i - p.w - c0 - 32 * q;          // columns >= lo are inside the window
-                    keep |= lo <= 0 ? 0xffffffffu : (lo >= 32 ? 0u : ~((1u << (int)lo) - 1u));
+                    const uint32_t win = lo <= 0 ? 0xffffffffu : (lo >= 32 ? 0u : ~((1u << (int)lo) - 1u));
+                    keep = p.local_only ? (win & ~keep) : (keep | win);     // window pass: in the window and not sharing
                 }
             }
             if (need_causal) {
@@ -911,7 +917,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
             if (!ctl_wait(&ctl.o_full[x], it & 1, &ctl)) { report_timeout(p, &ctl, 40 + x, (int)item); break; }
             tc_fence_after();
-            const float inv_l = 1.f / l;
+            const float inv_l = l > 0.f ? 1.f / l : 0.f;        // a row without any pair (possible in a partial pass): zeros, lse = -inf
             __nv_bfloat16* orow = p.o + (size_t)bb * p.o_sb + (size_t)h * p.o_sh + (size_t)(valid ? i : 0) * p.o_sn +
                                   half * (D / 2);
 #pragma unroll 1
@@ -919,7 +925,14 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 uint32_t ov[32];
                 tmem_ld32(t_o + c * 32, ov);
                 tmem_wait_ld();
-                if (valid) {
+                if (valid && p.o32) {
+                    float* o32row = p.o32 + ((size_t)hq * p.n + (size_t)i) * D + half * (D / 2) + c * 32;
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4)
+                        *reinterpret_cast<float4*>(o32row + e) =
+                            make_float4(__uint_as_float(ov[e]) * inv_l, __uint_as_float(ov[e + 1]) * inv_l,
+                                        __uint_as_float(ov[e + 2]) * inv_l, __uint_as_float(ov[e + 3]) * inv_l);
+                } else if (valid) {
 #pragma unroll
                     for (int e = 0; e < 32; e += 8) {
                         uint4 w4;
@@ -947,7 +960,8 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
     using C = AttnCfg<D, GATE>;
     CUtensorMap tq, tk, tv;
     int rc;
-    const bool sorted = a.ws && a.L.layout == FOCUS_LAYOUT_CLASS_SORTED;
+    const bool sorted = a.ws && !a.local_pass &&
+                        (a.L.layout == FOCUS_LAYOUT_CLASS_SORTED || a.L.layout == FOCUS_LAYOUT_SORTED_LOCAL);
     if (sorted) {
         // gather Q, K, V into the sorted order kept in the workspace; the kernel reads the copies
         char* ws = const_cast<char*>(a.ws);
@@ -993,6 +1007,8 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
     p.order = sorted ? reinterpret_cast<const int32_t*>(a.ws + a.L.order) : nullptr;
     p.counters = a.ws ? reinterpret_cast<const unsigned long long*>(a.ws + a.L.counters) : nullptr;
     p.gate_g = a.gate_g; p.gate_ld = a.gate_ld; p.gate_hl = 0.5f * a.gate_lambda;
+    p.local_only = a.local_pass ? 1 : 0;
+    p.o32 = a.o32;
     if (sorted) p.nitems = (long long)a.s.batch * a.s.Hq * p.nqblk * p.ipb;
     int dev = 0, sms = 0;
     if ((rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice"))) return rc;
@@ -1006,7 +1022,30 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
     return check_cuda(cudaGetLastError(), "attention kernel launch");
 }
 
+static int launch_attn_one(const AttnArgs& a, cudaStream_t st);
+
 int launch_attn_sm100(const AttnArgs& a, cudaStream_t st) {
+    if (a.ws && a.L.layout == FOCUS_LAYOUT_SORTED_LOCAL && !a.local_pass) {
+        // (1) sharing pairs in the class-sorted order -> o, lse; rows of blocks without key tiles keep lse = -inf
+        // (2) window-only pairs in token order -> workspace; (3) join through the logsumexps
+        char* ws = const_cast<char*>(a.ws);
+        const size_t rows = (size_t)a.s.batch * a.s.Hq * a.s.n;
+        int rc = launch_fill_f32(a.lse, rows, -INFINITY, st);
+        if (rc) return rc;
+        AttnArgs s1 = a;
+        s1.o32 = reinterpret_cast<float*>(ws + a.L.o_sorted);
+        if ((rc = launch_attn_one(s1, st))) return rc;
+        AttnArgs s2 = a;
+        s2.local_pass = true;
+        s2.o32 = reinterpret_cast<float*>(ws + a.L.o_local);
+        s2.lse = reinterpret_cast<float*>(ws + a.L.lse_local);
+        if ((rc = launch_attn_one(s2, st))) return rc;
+        return launch_merge_partials(&a.s, a.o, a.lse, s1.o32, s2.o32, s2.lse, st);
+    }
+    return launch_attn_one(a, st);
+}
+
+static int launch_attn_one(const AttnArgs& a, cudaStream_t st) {
     const bool cap = a.s.softcap > 0.f;
     if (a.gate_g) {      // training-time gated forward: dense causal walk, no softcap
         switch (a.s.D) {

@@ -57,6 +57,10 @@ int launch_build_tiles(const focus_shape* s, const uint32_t* mq, const uint32_t*
 // class-sorted layout: copy the rows of t into the sorted order of the workspace (query or key side)
 int launch_gather_sorted(const focus_shape* s, const focus_tensor& t, int H, bool query, const focus_tiles_layout& L,
                          const char* ws, char* dst, cudaStream_t st);
+int launch_fill_f32(float* x, size_t count, float v, cudaStream_t st);
+// FOCUS_LAYOUT_SORTED_LOCAL: the partial results of the class-sorted pass (o_sorted, lse) and of the window pass are joined into o, lse
+int launch_merge_partials(const focus_shape* s, const focus_tensor& o, float* lse, const float* o_sorted, const float* o_local,
+                          const float* lse_local, cudaStream_t st);
 int launch_count_kept(const focus_shape* s, const uint32_t* mq, const focus_tiles_layout& L, const char* ws,
                       unsigned long long* out, cudaStream_t st);
 
@@ -70,6 +74,8 @@ struct AttnArgs {
     float* lse;
     int32_t* dev_status;
     float scale;              // resolved logit scale
+    float* o32 = nullptr;            // when set, O goes there in fp32, rows [batch*Hq][n][D], instead of to `o` (partial passes)
+    bool local_pass = false;         // FOCUS_LAYOUT_SORTED_LOCAL: the window pass in token order (pairs without a shared group)
     const float* gate_g = nullptr;   // training-time soft gate: assignments [batch, n, gate_ld]; nullptr = no gate
     int gate_ld = 0;
     float gate_lambda = 0.f;

@@ -196,7 +196,7 @@ qrange_kernel(int HQ, int Hq, int Hkv, int G_heads, int w, int nqp, int nkp, con
               const int32_t* __restrict__ ncls_k, const uint32_t* __restrict__ cls_q, const uint32_t* __restrict__ cls_k,
               const int32_t* __restrict__ cnt_q, const int32_t* __restrict__ cnt_k, const int32_t* __restrict__ seg_q,
               const int32_t* __restrict__ seg_k, const int32_t* __restrict__ perm_q, const int32_t* __restrict__ perm_k,
-              int32_t* __restrict__ qrange, int32_t* __restrict__ cost, unsigned long long* counters) {
+              int32_t* __restrict__ qrange, int32_t* __restrict__ cost, unsigned long long* counters, int sharing_only) {
     const int nqblk = nqp / 256;
     const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (gid >= (long long)HQ * nqblk * MAXC) return;
@@ -219,7 +219,8 @@ qrange_kernel(int HQ, int Hq, int Hkv, int G_heads, int w, int nqp, int nkp, con
         const bool share = (cls_q[(size_t)hq * MAXC + jq] & cls_k[(size_t)hk * MAXC + jk]) != 0u;
         const int hi = count_le(pk, kc, pmax);                             // keys at or before the block's last position
         const int lo = share ? 0 : count_le(pk, kc, pmin - w - 1);          // keys before the window of the first row
-        if (hi > lo) {
+        // with a separate window pass only the classes that share a group with the block's class are listed
+        if (hi > lo && (share || !sharing_only)) {
             first = (ks0 + lo) / 128;
             last = (ks0 + hi + 127) / 128;
         }
@@ -373,10 +374,91 @@ int launch_build_tiles_sorted(const focus_shape* s, const uint32_t* mq, const ui
         reinterpret_cast<const uint32_t*>(ws + L.cls_k), reinterpret_cast<const int32_t*>(ws + L.cnt_q),
         reinterpret_cast<const int32_t*>(ws + L.cnt_k), reinterpret_cast<const int32_t*>(ws + L.seg_q),
         reinterpret_cast<const int32_t*>(ws + L.seg_k), reinterpret_cast<const int32_t*>(ws + L.perm_q),
-        reinterpret_cast<const int32_t*>(ws + L.perm_k), reinterpret_cast<int32_t*>(ws + L.qrange), cost, counters);
+        reinterpret_cast<const int32_t*>(ws + L.perm_k), reinterpret_cast<int32_t*>(ws + L.qrange), cost, counters,
+        L.layout == FOCUS_LAYOUT_SORTED_LOCAL ? 1 : 0);
     order_kernel<<<HK, 1024, 0, st>>>(s->Hq, s->Hkv, s->Hq / s->Hkv, nqblk, L.nkp / 128, cost,
                                       reinterpret_cast<int32_t*>(ws + L.order));
     return check_cuda(cudaGetLastError(), "build_tiles (class-sorted) kernels");
+}
+
+// ---- FOCUS_LAYOUT_SORTED_LOCAL: the two partial results (sharing pairs from the class-sorted pass, window-only pairs
+// from the pass in token order) cover disjoint sets of pairs and join through their logsumexps (paper Appendix C).
+
+__global__ void __launch_bounds__(256) fill_f32_kernel(float* __restrict__ x, size_t count, float v) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < count) x[i] = v;
+}
+
+int launch_fill_f32(float* x, size_t count, float v, cudaStream_t st) {
+    fill_f32_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(x, count, v);
+    return check_cuda(cudaGetLastError(), "fill kernel launch");
+}
+
+// thread = 8 consecutive elements of a row; the D/8 threads of a row sit in one warp, so that all of them have read the
+// row's two logsumexps before the first of them overwrites one
+template <int D>
+__global__ void __launch_bounds__(256)
+merge_partials_kernel(__nv_bfloat16* __restrict__ o, int64_t o_sb, int64_t o_sh, int64_t o_sn, float* __restrict__ lse,
+                      const float* __restrict__ o_sorted, const float* __restrict__ o_local, const float* __restrict__ lse_local,
+                      int Hq, int n) {
+    constexpr int TPR = D / 8;
+    const int hq = blockIdx.y;
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long i = t / TPR;
+    const int c = (int)(t % TPR);
+    const bool in = i < n;
+    float ls = -INFINITY, ll = -INFINITY;
+    if (in) {
+        ls = lse[(size_t)hq * n + i];
+        ll = lse_local[(size_t)hq * n + i];
+    }
+    __syncwarp();
+    if (!in) return;
+    const float m = fmaxf(ls, ll);
+    const float ws = m == -INFINITY ? 0.f : __expf(ls - m), wl = m == -INFINITY ? 0.f : __expf(ll - m);
+    const float tot = ws + wl;
+    const float inv = tot > 0.f ? 1.f / tot : 0.f;
+    const size_t src = ((size_t)hq * n + i) * D + c * 8;
+    float r[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) r[e] = 0.f;
+    // a partial result without any pair has weight 0 and unspecified contents: it is not read
+    if (ws > 0.f) {
+        const float4 a0 = *reinterpret_cast<const float4*>(o_sorted + src), a1 = *reinterpret_cast<const float4*>(o_sorted + src + 4);
+        const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) r[e] = av[e] * ws;
+    }
+    if (wl > 0.f) {
+        const float4 b0 = *reinterpret_cast<const float4*>(o_local + src), b1 = *reinterpret_cast<const float4*>(o_local + src + 4);
+        const float bv[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) r[e] = fmaf(bv[e], wl, r[e]);
+    }
+    uint32_t rw[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat162 h2 = __floats2bfloat162_rn(r[2 * e] * inv, r[2 * e + 1] * inv);
+        rw[e] = *reinterpret_cast<const uint32_t*>(&h2);
+    }
+    __nv_bfloat16* orow = o + (size_t)(hq / Hq) * o_sb + (size_t)(hq % Hq) * o_sh + (size_t)i * o_sn + c * 8;
+    *reinterpret_cast<uint4*>(orow) = make_uint4(rw[0], rw[1], rw[2], rw[3]);
+    if (c == 0) lse[(size_t)hq * n + i] = tot > 0.f ? m + __logf(tot) : -INFINITY;
+}
+
+int launch_merge_partials(const focus_shape* s, const focus_tensor& o, float* lse, const float* o_sorted, const float* o_local,
+                          const float* lse_local, cudaStream_t st) {
+    const int HQ = s->batch * s->Hq;
+    const long long threads = (long long)s->n * (s->D / 8);
+    const dim3 grid((unsigned)((threads + 255) / 256), HQ);
+    auto* op = reinterpret_cast<__nv_bfloat16*>(o.ptr);
+    switch (s->D) {
+        case 64: merge_partials_kernel<64><<<grid, 256, 0, st>>>(op, o.stride_b, o.stride_h, o.stride_n, lse, o_sorted, o_local, lse_local, s->Hq, s->n); break;
+        case 128: merge_partials_kernel<128><<<grid, 256, 0, st>>>(op, o.stride_b, o.stride_h, o.stride_n, lse, o_sorted, o_local, lse_local, s->Hq, s->n); break;
+        case 256: merge_partials_kernel<256><<<grid, 256, 0, st>>>(op, o.stride_b, o.stride_h, o.stride_n, lse, o_sorted, o_local, lse_local, s->Hq, s->n); break;
+        default: return fail(FOCUS_ERR_UNSUPPORTED, "D (%d) must be 64, 128 or 256", s->D);
+    }
+    return check_cuda(cudaGetLastError(), "merge kernel launch");
 }
 
 }  // namespace focus

@@ -103,13 +103,18 @@ def test_auto_layout_is_resolved_from_the_shape():
     pick = lambda Hq, Hkv, n, K, t: fb.focus_tiles_layout_of(fb.make_shape(Hq, Hkv, n, 128, K, t, 2048), fb.FOCUS_LAYOUT_AUTO).layout
     assert pick(32, 8, 8192, 4, 1) == 0 and pick(32, 8, 16384, 4, 1) == 1          # top-1 of 4: 3/4 of far pairs fall away
     assert pick(32, 8, 32768, 4, 2) == 0 and pick(32, 8, 131072, 4, 2) == 1        # top-2 of 4: only 1/6 fall away
-    assert pick(32, 8, 16384, 8, 1) == 1
-    assert pick(32, 8, 32768, 8, 2) == 0 and pick(32, 8, 65536, 8, 2) == 1         # 28 classes need 2048 tokens each
+    # many classes: the window of a sorted query block is spread over 7 (or 15) other classes -> separate window pass
+    assert pick(32, 8, 16384, 8, 1) == 3
+    assert pick(32, 8, 32768, 8, 2) == 0 and pick(32, 8, 65536, 8, 2) == 3         # 28 classes need 2048 tokens each
     assert pick(4, 2, 1 << 20, 32, 3) == 0                                          # more classes than the sorted layout holds
     s = fb.make_shape(32, 8, 131072, 128, 4, 2, 2048)
     assert fb.focus_tiles_workspace_bytes(s, fb.FOCUS_LAYOUT_AUTO) == fb.focus_tiles_workspace_bytes(s, 1)
     L = fb.focus_tiles_layout()
-    assert fb.lib().focus_tiles_layout_of(ctypes.byref(s), 3, ctypes.byref(L)) == -1
+    assert fb.lib().focus_tiles_layout_of(ctypes.byref(s), 4, ctypes.byref(L)) == -1
+    # the split layout: the sorted arrays plus two fp32 partial results and one logsumexp per row
+    L1, L3 = fb.focus_tiles_layout_of(s, 1), fb.focus_tiles_layout_of(s, 3)
+    assert L3.layout == 3 and L3.qrange == L1.qrange and L1.o_sorted == 0 and L3.o_sorted >= L1.total_bytes
+    assert L3.o_local - L3.o_sorted >= 32 * 131072 * 128 * 4 and L3.total_bytes - L3.lse_local >= 32 * 131072 * 4
 
 
 def test_training_forward_host_checks():

@@ -162,6 +162,7 @@ def test_cfg2_sorted_two_heads_all_rows_others_sampled():
 
 def test_auto_layout_runs_whichever_it_picks():
     for wl, expect in ((fi.Workload("a0", 4, 2, 128, 3000, 4, 1, 64, seed=51), 0),
-                       (fi.Workload("a1", 4, 2, 128, 17000, 4, 1, 64, seed=52), 1)):
+                       (fi.Workload("a1", 4, 2, 128, 17000, 4, 1, 64, seed=52), 1),
+                       (fi.Workload("a3", 4, 2, 128, 17000, 8, 1, 512, seed=53), 3)):
         assert fb.focus_tiles_layout_of(fb.shape_of(wl), fb.FOCUS_LAYOUT_AUTO).layout == expect
         run_case(wl, layout=fb.FOCUS_LAYOUT_AUTO, rows=fi.sample_rows(wl, 200))
