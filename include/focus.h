@@ -75,8 +75,8 @@ typedef struct {
 #define FOCUS_LAYOUT_ORIGINAL 0
 #define FOCUS_LAYOUT_CLASS_SORTED 1
 /* Let the library choose from the shape alone (n, K, topk, window): a class-sorted layout when the
- * sequence is long enough for its fixed costs (at least 16384 tokens and 2048 per mask class, C(K, topk) classes
- * assumed) and enough distant pairs fall away (at least half of them for uniform memberships, or at least 15 % from
+ * sequence is long enough for its fixed costs (at least 16384 tokens and 2048 per mask class, 1024 with the separate
+ * window pass; C(K, topk) classes assumed) and enough distant pairs fall away (at least half of them for uniform memberships, or at least 15 % from
  * 65536 tokens on); the original layout otherwise.  Of the two class-sorted layouts FOCUS_LAYOUT_SORTED_LOCAL is taken
  * when the window of a block of sorted queries, spread over the C(K-topk, topk) classes it shares no group with,
  * would cost over 1.25 times the key tiles of a window pass in token order, fixed costs included (many classes: K = 8).

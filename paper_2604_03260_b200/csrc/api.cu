@@ -80,19 +80,20 @@ static int choose_layout(const focus_shape* s) {
     const double classes = binom(s->K, s->topk);
     if (classes > (double)FOCUS_MAX_CLASSES + 0.5) return FOCUS_LAYOUT_ORIGINAL;
     const double dropped = binom(s->K - s->topk, s->topk) / classes;      // far pairs without a shared group, uniform memberships
-    const double min_n = classes * 2048.0 > 16384.0 ? classes * 2048.0 : 16384.0;
+    // Which of the two class-sorted layouts.  Key tiles a block of 256 sorted queries visits for its window alone: its
+    // rows span about 256 * classes positions, so the window of the block covers (256 * classes + w) / classes keys of
+    // every class that shares no group with it.  The separate window pass in token order reads w + 256 keys once per
+    // 256 rows, plus what a second pass costs per block whatever its length (query load, pipeline fill, fp32 partial
+    // results, merge): about six key tiles' worth, measured.  The pass is taken when it saves a quarter or more.
+    const double apart = binom(s->K - s->topk, s->topk);                 // classes without a shared group
+    const double in_sorted = apart * ((256.0 * classes + s->window) / classes / 128.0 + 1.0);
+    const double in_order = (s->window + 256.0) / 128.0 + 7.0;
+    const int sorted = in_sorted > 1.25 * in_order ? FOCUS_LAYOUT_SORTED_LOCAL : FOCUS_LAYOUT_CLASS_SORTED;
+    // long enough for the fixed costs of sorting: 2048 tokens per class, 1024 when the window has its own pass
+    const double per_class = sorted == FOCUS_LAYOUT_SORTED_LOCAL ? 1024.0 : 2048.0;
+    const double min_n = classes * per_class > 16384.0 ? classes * per_class : 16384.0;
     if ((double)s->n < min_n) return FOCUS_LAYOUT_ORIGINAL;
-    if (dropped >= 0.5 || (s->n >= 65536 && dropped >= 0.15)) {
-        // Key tiles a block of 256 sorted queries visits for its window alone: its rows span about 256 * classes
-        // positions, so the window of the block covers (256 * classes + w) / classes keys of every class that shares
-        // no group with it.  The separate window pass in token order reads w + 256 keys once per 256 rows, plus what
-        // a second pass costs per block whatever its length (query load, pipeline fill, fp32 partial results, merge):
-        // about six key tiles' worth, measured.  The pass is taken when it saves a quarter or more.
-        const double apart = binom(s->K - s->topk, s->topk);                 // classes without a shared group
-        const double in_sorted = apart * ((256.0 * classes + s->window) / classes / 128.0 + 1.0);
-        const double in_order = (s->window + 256.0) / 128.0 + 7.0;
-        return in_sorted > 1.25 * in_order ? FOCUS_LAYOUT_SORTED_LOCAL : FOCUS_LAYOUT_CLASS_SORTED;
-    }
+    if (dropped >= 0.5 || (s->n >= 65536 && dropped >= 0.15)) return sorted;
     return FOCUS_LAYOUT_ORIGINAL;
 }
 

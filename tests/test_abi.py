@@ -105,7 +105,7 @@ def test_auto_layout_is_resolved_from_the_shape():
     assert pick(32, 8, 32768, 4, 2) == 0 and pick(32, 8, 131072, 4, 2) == 1        # top-2 of 4: only 1/6 fall away
     # many classes: the window of a sorted query block is spread over 7 (or 15) other classes -> separate window pass
     assert pick(32, 8, 16384, 8, 1) == 3
-    assert pick(32, 8, 32768, 8, 2) == 0 and pick(32, 8, 65536, 8, 2) == 3         # 28 classes need 2048 tokens each
+    assert pick(32, 8, 16384, 8, 2) == 0 and pick(32, 8, 32768, 8, 2) == 3         # 28 classes need 1024 tokens each there
     assert pick(4, 2, 1 << 20, 32, 3) == 0                                          # more classes than the sorted layout holds
     s = fb.make_shape(32, 8, 131072, 128, 4, 2, 2048)
     assert fb.focus_tiles_workspace_bytes(s, fb.FOCUS_LAYOUT_AUTO) == fb.focus_tiles_workspace_bytes(s, 1)
