@@ -209,7 +209,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="focus", choices=["focus", "reference"])
     ap.add_argument("--workload", default="M128k")
-    ap.add_argument("--layout", type=int, default=1, help="0 = original token order, 1 = class-sorted (group-permuted), 2 = chosen by the library from the shape, "
+    ap.add_argument("--layout", type=int, default=2, help="0 = original token order, 1 = class-sorted (group-permuted), 2 = chosen by the library from the shape, "
                                                            "3 = class-sorted for sharing pairs + window pass in token order")
     ap.add_argument("--ref-rows", type=int, default=2048, help="oracle rows per step (reference arm)")
     ap.add_argument("--cpu-rows", type=int, default=24576, help="oracle rows of the cpu_baseline sample")
