@@ -107,7 +107,7 @@ typedef struct {
     size_t live;       /* uint32 [B*Hq][nqt][nkw]: bit b set when (a, b) is a far tile pair that may hold a kept pair */
     size_t live_cnt;   /* int32  [B*Hq][nqt]: popcount of the row of `live` */
     size_t kany, kall; /* uint32 [B*Hkv][K][nkw]: bit b set when key tile b holds a member of group g / only members of g */
-    /* class-sorted layout only (0 otherwise) */
+    /* class-sorted layouts only (0 otherwise) */
     int32_t nqp, nkp;  /* capacity of the sorted arrays in rows (multiples of 256): n + room for padding every class segment */
     size_t ncls_q, ncls_k;   /* int32 [B*Hq], [B*Hkv]: distinct mask values of the head */
     size_t cls_q, cls_k;     /* uint32 [heads][FOCUS_MAX_CLASSES]: the mask values, ascending */
@@ -189,7 +189,9 @@ FOCUS_API size_t focus_tiles_workspace_bytes(const focus_shape* shape, int32_t l
  * OR(query tile masks) & OR(key tile masks) != 0; dead far pairs hold no attended pair.
  *   mq   device, uint32 [batch*Hq, n]    mk   device, uint32 [batch*Hkv, n]
  *   layout  FOCUS_LAYOUT_ORIGINAL, or FOCUS_LAYOUT_CLASS_SORTED (tokens stably sorted by mask value
- *           per head, so that a tile holds one mask class and tile pairs are all-share or none-share)
+ *           per head, so that a tile holds one mask class and tile pairs are all-share or none-share),
+ *           or FOCUS_LAYOUT_SORTED_LOCAL (the same arrays, with only the sharing classes listed in `qrange`),
+ *           or FOCUS_LAYOUT_AUTO
  *   ws   device workspace of ws_bytes >= focus_tiles_workspace_bytes(shape, layout), 256-byte aligned.
  *        Contents are described by focus_tiles_layout.  The workspace is tied to (shape, mq, mk).
  */
