@@ -168,3 +168,27 @@ def test_chain_hidden_to_gated_output():
     err = np.abs(O[0].float().cpu().numpy() - refO)
     assert err.max() <= O_MAX_ABS and err.mean() <= O_MEAN_ABS
     assert np.abs(lse[0].cpu().numpy() - refL).max() <= LSE_MAX_ABS
+
+
+def test_gated_attention_at_the_metric_point_shape():
+    """32 / 8 heads, D = 128, 131072 tokens, K = 4, w = 2048 (the launch the bench times): sampled rows of every head"""
+    n, K, w, lam = 131072, 4, 2048, 10.0
+    Q, Kt, V, gt = gate_case(32, 8, n, 128, K, 61)
+    O, lse = run_gate(Q, Kt, V, gt, K, w, lam)
+    rng = np.random.default_rng(4)
+    rows = np.unique(np.concatenate([rng.integers(0, n, 6), [0, w, w + 1, n // 2, n - 1]]))
+    check_gate(Q, Kt, V, gt, K, w, lam, O, lse, rows)
+
+
+def test_sinkhorn_one_million_tokens():
+    n, K, tau, iters = 1 << 20, 8, 0.1, 10
+    g = torch.Generator(device="cuda"); g.manual_seed(8)
+    S = padded(0.3 * torch.randn((1, n, K), generator=g, device="cuda"), 8)
+    shape = fb.make_shape(32, 8, n, 128, K, 1, 2048)
+    ws = torch.empty(fb.focus_sinkhorn_workspace_bytes(shape, iters), dtype=torch.uint8, device="cuda")
+    out = torch.empty_like(S)
+    fb.focus_sinkhorn(shape, S, tau, iters, ws, out)
+    torch.cuda.synchronize()
+    ref = fo.sinkhorn(S[0].cpu().numpy().astype(np.float64), tau, iters)
+    np.testing.assert_allclose(out[0].cpu().numpy(), ref, rtol=5e-4, atol=1e-7)
+    np.testing.assert_allclose(out[0].sum(dim=0).cpu().numpy(), n / K, rtol=2e-2)      # groups close to balanced after 10 iterations
