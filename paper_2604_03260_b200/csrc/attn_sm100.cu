@@ -149,7 +149,6 @@ struct TileWalk {
             if (nq > 1 && a0 + 1 < p.nqt) l1 = l0 + p.nkw;
         }
         far_phase = f0 > 0 && !p.local_only;
-        jk = 0;
         wd = -1;
         bits = 0;
         b = f0;
@@ -345,7 +344,8 @@ __device__ __forceinline__ int count_le_128(const int32_t* __restrict__ a, int v
 // "no mask needed" / "nothing attended" are taken per warp from the warp's smallest and largest row
 // position.
 __device__ __forceinline__ void build_tile_mask_sorted(TileMask& tm, int w, const int32_t* __restrict__ kpos, bool share,
-                                                       int pos, int wmin, int wmax, int k_first, int k_last) {
+                                                       int pos, int wmin, int wmax) {
+    const int k_first = __ldg(kpos), k_last = __ldg(kpos + 127);
     tm.all_masked = wmax < 0 || k_first > wmax;
     const bool need_causal = k_last > wmin;
     const bool need_window = !share && ((long long)wmax - k_first > w);
@@ -713,28 +713,12 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     }
                 }
             }
-            // class-sorted layout: the class word and the first and last position of a tile are fetched one tile ahead,
-            // so that their latency is not added to the S -> P chain of the tile they belong to
-            uint32_t pf_cls = 0;
-            int pf_first = 0, pf_last = 0;
-            auto prefetch = [&](int tile, int jk) {
-                if (p.sorted && tile >= 0) {
-                    const int32_t* kp = p.perm_k + (size_t)hk * p.nkp + (size_t)tile * 128;
-                    pf_cls = __ldg(p.cls_k + (size_t)hk * FOCUS_MAX_CLASSES + jk);
-                    pf_first = __ldg(kp);
-                    pf_last = __ldg(kp + 127);
-                }
-            };
-            prefetch(kb, walk.jk);
-            for (int nkb; kb >= 0; kb = nkb) {
-                const uint32_t cur_cls = pf_cls;
-                const int cur_first = pf_first, cur_last = pf_last;
-                nkb = walk.next();
-                prefetch(nkb, walk.jk);
+            for (; kb >= 0; kb = walk.next()) {
                 TileMask tm;
                 if (p.sorted) {
-                    build_tile_mask_sorted(tm, p.w, p.perm_k + (size_t)hk * p.nkp + (size_t)kb * 128, (mi & cur_cls) != 0u,
-                                           valid ? (int)i : -1, wmin, wmax, cur_first, cur_last);
+                    const bool share = (mi & __ldg(p.cls_k + (size_t)hk * FOCUS_MAX_CLASSES + walk.jk)) != 0u;
+                    build_tile_mask_sorted(tm, p.w, p.perm_k + (size_t)hk * p.nkp + (size_t)kb * 128, share,
+                                           valid ? (int)i : -1, wmin, wmax);
                 } else {
                     build_tile_mask(tm, p, a, kb, i, mi, aq, f_x, hk);
                 }
@@ -827,53 +811,6 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         for (int c = 0; c < NC; ++c)
                             sr[c] = ((tm.kw[(NSPLIT == 2 ? half * 2 : 0) + (c >> 5)] >> (c & 31)) & 1u) ? sr[c] : 0xff800000u;      // -inf
                     }
-                    // ---- once every row of the warp has a reference maximum, the exponentials start at once against that
-                    // reference and the tile's row maximum is taken on the side, off the S -> P chain.  The reference may lag
-                    // by the rescale threshold anyway; when some row's maximum has outrun it by more, the probabilities are
-                    // thrown away, S is read again (P has not been stored over it yet) and the tile goes the long way.
-                    bool fast_done = false;
-                    if constexpr (NSPLIT == 1 && !GATE) {
-                        if (__all_sync(0xffffffffu, m_used != -INFINITY)) {
-                            const float2 sl2v = make_float2(sl2, sl2), nmv = make_float2(-m_used, -m_used);
-                            float2 acc[4];
-                            float fx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) acc[e] = make_float2(0.f, 0.f);
-#pragma unroll
-                            for (int c = 0; c < NC; c += 8) {
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const float s0 = __uint_as_float(sr[c + 2 * e]), s1 = __uint_as_float(sr[c + 2 * e + 1]);
-                                    const float2 xv = __ffma2_rn(make_float2(s0, s1), sl2v, nmv);
-                                    float2 pr;
-                                    pr.x = ex2_approx(xv.x);
-                                    pr.y = ex2_approx(xv.y);
-                                    acc[e] = __fadd2_rn(acc[e], pr);
-                                    pk[(c >> 1) + e] = pack_bf16x2(pr.x, pr.y);
-                                    fx[e] = max3(fx[e], s0, s1);
-                                }
-                            }
-                            const float mt = max3(fx[0], fx[1], fmaxf(fx[2], fx[3])) * sl2;
-                            if (!__any_sync(0xffffffffu, mt > m_used + RESCALE_THRESHOLD)) {
-                                l += (acc[0].x + acc[0].y) + (acc[1].x + acc[1].y) + ((acc[2].x + acc[2].y) + (acc[3].x + acc[3].y));
-                                fast_done = true;
-                            } else {
-#pragma unroll
-                                for (int c = 0; c < NC / 32; ++c) tmem_ld32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[c * 32]));
-                                tmem_wait_ld();
-                                if (SOFTCAP) {
-#pragma unroll
-                                    for (int c = 0; c < NC; ++c) sr[c] = __float_as_uint(tanh_approx(__uint_as_float(sr[c]) * cap_in));
-                                }
-                                if (tm.masked) {
-#pragma unroll
-                                    for (int c = 0; c < NC; ++c)
-                                        sr[c] = ((tm.kw[c >> 5] >> (c & 31)) & 1u) ? sr[c] : 0xff800000u;
-                                }
-                            }
-                        }
-                    }
-                    if (!fast_done) {
                     // ---- row maximum of the tile: four independent chains of three-input maxima
                     float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
@@ -948,7 +885,6 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         }
                     }
                     l += (acc[0].x + acc[0].y) + (acc[1].x + acc[1].y) + ((acc[2].x + acc[2].y) + (acc[3].x + acc[3].y));
-                    }   // !fast_done
                 }
 #pragma unroll
                 for (int c = 0; c < NC / 64; ++c) tmem_st32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[c * 32]));
