@@ -215,9 +215,13 @@ FOCUS_API int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, co
  *               class-sorted order kept in the workspace, walks only sharing class pairs plus the
  *               window, and scatters O/lse back to token order.
  *   lse         device fp32 [batch*Hq, n], natural log
- *   dev_status  device int32[4], nullable: [0] is set non-zero if a bounded wait inside the kernel
- *               expired (the kernel then drains and exits; outputs are invalid), [1..3] say where.
- *               The caller zeroes it and reads it after synchronising.
+ *   dev_status  device int32[4], nullable: [0] stays 0 on success.  [0] = 1: a bounded wait inside the
+ *               kernel expired (the kernel then drains and exits; outputs are invalid), [1] = code of
+ *               the wait, [2] = work item, [3] = CTA.  [0] = 2: a class-sorted layout was asked for
+ *               but a head holds more than FOCUS_MAX_CLASSES distinct mask values (possible only with
+ *               masks that do not come from a top-k rule); nothing was computed and O / lse were not
+ *               written.  Pass a non-NULL dev_status with layouts 1 and 3 when the masks are not the
+ *               library's own.  The caller zeroes it and reads it after synchronising.
  */
 FOCUS_API int focus_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k, focus_tensor v,
                    const uint32_t* mq, const uint32_t* mk, const void* tiles_ws, int32_t layout,
@@ -266,8 +270,11 @@ FOCUS_API int focus_count_kept(const focus_shape* shape, const uint32_t* mq, con
  * Limit: batch*Hkv*ceil(n/128)*K*16 bytes must fit in FOCUS_NOALLOC_MAX_BYTES, otherwise
  * FOCUS_ERR_CAPACITY is returned and nothing is launched (1 MiB covers the 128K-token metric point:
  * 8 KV heads x 1024 tiles x 4 groups x 16 B = 512 KiB).
- * The first call on each device looks up the array's device address (with that device current);
- * make that first call outside any stream capture.  All calls share the one array, which keeps the
+ * batch*Hq and batch*Hkv must not exceed 65535 (FOCUS_ERR_UNSUPPORTED otherwise, nothing launched).
+ * The first call on each device looks up the array's device address (with that device current)
+ * and keeps it for the life of the process; make that first call outside any stream capture, and
+ * do not call this entry point again on a device whose context the application has destroyed
+ * (cudaDeviceReset): the remembered address is then stale.  All calls share the one array, which keeps the
  * previous call's contents; each call rewrites the part it reads, so stale contents are harmless,
  * but two calls whose kernels may overlap on the GPU (different streams) race on it.
  */

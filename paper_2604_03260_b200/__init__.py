@@ -4,4 +4,4 @@ The work is done by a C-ABI CUDA library (``csrc/``, declared in ``include/focus
 is its thin ctypes binding plus the seeded input generators.  Importing the package does not load
 the library; ``paper_2604_03260_b200.binding`` does, and fails loudly when it is missing.
 """
-__all__ = ["inputs", "binding", "build"]
+__all__ = ["inputs", "binding", "build", "host_pipeline", "multi"]

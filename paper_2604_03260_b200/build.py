@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfocus_b200.so")
-SOURCES = ["api.cu", "assign.cu", "assign_hidden.cu", "sinkhorn.cu", "decode.cu", "tiles.cu", "tiles_sorted.cu", "attn_simple.cu", "attn_sm100.cu", "selftest.cu",
+SOURCES = ["api.cu", "assign.cu", "assign_hidden.cu", "sinkhorn.cu", "decode.cu", "tiles.cu", "tiles_sorted.cu", "attn_sm100.cu", "selftest.cu",
            "tma_host.cu", "noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]

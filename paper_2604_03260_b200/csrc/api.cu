@@ -45,10 +45,14 @@ int validate_shape(const focus_shape* s) {
     return FOCUS_OK;
 }
 
-int validate_tensor(const char* name, const focus_tensor& t, bool tma) {
+int validate_tensor(const char* name, const focus_tensor& t, bool tma, int batch) {
     if (!t.ptr) return fail(FOCUS_ERR_INVALID_ARG, "%s.ptr is NULL", name);
     if (t.stride_n < 1 || t.stride_h < 1 || t.stride_b < 0)
         return fail(FOCUS_ERR_INVALID_ARG, "%s has a non-positive stride", name);
+    // a batch stride of 0 is accepted as "unused" for a single sequence only: with batch > 1 it would
+    // alias every sequence onto the first one
+    if (batch > 1 && t.stride_b < 1)
+        return fail(FOCUS_ERR_INVALID_ARG, "%s.stride_b must be positive when batch > 1", name);
     if (tma) {
         if ((uintptr_t)t.ptr % 16) return fail(FOCUS_ERR_INVALID_ARG, "%s.ptr is not 16-byte aligned", name);
         if (t.stride_n % 8 || t.stride_h % 8 || t.stride_b % 8)
@@ -189,7 +193,7 @@ int focus_assign(const focus_shape* shape, focus_tensor x, int32_t H, const floa
     int rc = validate_shape(shape);
     if (rc) return rc;
     if (H != shape->Hq && H != shape->Hkv) return fail(FOCUS_ERR_INVALID_ARG, "H (%d) must be Hq or Hkv", H);
-    if ((rc = validate_tensor("x", x, false))) return rc;
+    if ((rc = validate_tensor("x", x, false, shape->batch))) return rc;
     if ((uintptr_t)x.ptr % 16 || x.stride_n % 8 || x.stride_h % 8 || x.stride_b % 8)
         return fail(FOCUS_ERR_INVALID_ARG, "x must be 16-byte aligned with strides that are multiples of 8 elements");
     if (!centroids || !masks_out) return fail(FOCUS_ERR_INVALID_ARG, "centroids or masks_out is NULL");
@@ -283,7 +287,13 @@ int focus_decode_step(const focus_shape* shape, focus_tensor q, focus_tensor k, 
     int rc = validate_shape(shape);
     if (rc) return rc;
     if (!q.ptr || !o.ptr || !mq_new || !mk || !lse || !ws) return fail(FOCUS_ERR_INVALID_ARG, "a pointer argument is NULL");
-    if ((rc = validate_tensor("k", k, true)) || (rc = validate_tensor("v", v, true))) return rc;
+    if ((rc = validate_tensor("k", k, true, shape->batch)) || (rc = validate_tensor("v", v, true, shape->batch))) return rc;
+    // the query vectors are read two elements at a time
+    if ((uintptr_t)q.ptr % 4 || q.stride_h % 2 || q.stride_b % 2 || q.stride_h < 1 || o.stride_h < 1 || q.stride_b < 0 ||
+        o.stride_b < 0)
+        return fail(FOCUS_ERR_INVALID_ARG, "q must be 4-byte aligned with even, positive head strides (o: positive strides)");
+    if (shape->batch > 1 && (q.stride_b < 1 || o.stride_b < 1))
+        return fail(FOCUS_ERR_INVALID_ARG, "q.stride_b and o.stride_b must be positive when batch > 1");
     if ((uintptr_t)ws % 16) return fail(FOCUS_ERR_INVALID_ARG, "ws is not 16-byte aligned");
     if (ws_bytes < decode_workspace_bytes(shape))
         return fail(FOCUS_ERR_CAPACITY, "decode workspace has %zu bytes, %zu needed", ws_bytes, decode_workspace_bytes(shape));
@@ -307,8 +317,9 @@ int focus_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k, foc
                    int32_t* dev_status, void* stream) {
     int rc = validate_shape(shape);
     if (rc) return rc;
-    if ((rc = validate_tensor("q", q, true)) || (rc = validate_tensor("k", k, true)) ||
-        (rc = validate_tensor("v", v, true)) || (rc = validate_tensor("o", o, true)))
+    const int nb = shape->batch;
+    if ((rc = validate_tensor("q", q, true, nb)) || (rc = validate_tensor("k", k, true, nb)) ||
+        (rc = validate_tensor("v", v, true, nb)) || (rc = validate_tensor("o", o, true, nb)))
         return rc;
     if (!lse) return fail(FOCUS_ERR_INVALID_ARG, "lse is NULL");
     if (tiles_ws && (!mq || !mk)) return fail(FOCUS_ERR_INVALID_ARG, "mq/mk are required with a tiles workspace");
@@ -323,8 +334,6 @@ int focus_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k, foc
     a.scale = shape->scale > 0.f ? shape->scale : 1.0f / sqrtf((float)shape->D);
     memset(&a.L, 0, sizeof a.L);
     if (tiles_ws && (rc = layout_of(shape, layout, &a.L))) return rc;
-    const char* impl = getenv("FOCUS_ATTN_IMPL");
-    if (impl && !strcmp(impl, "simple")) return launch_attn_simple(a, (cudaStream_t)stream);
     return launch_attn_sm100(a, (cudaStream_t)stream);
 }
 
@@ -332,8 +341,9 @@ int focus_gate_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k
                         focus_tensor o, float* lse, int32_t* dev_status, void* stream) {
     int rc = validate_shape(shape);
     if (rc) return rc;
-    if ((rc = validate_tensor("q", q, true)) || (rc = validate_tensor("k", k, true)) ||
-        (rc = validate_tensor("v", v, true)) || (rc = validate_tensor("o", o, true)))
+    const int nb = shape->batch;
+    if ((rc = validate_tensor("q", q, true, nb)) || (rc = validate_tensor("k", k, true, nb)) ||
+        (rc = validate_tensor("v", v, true, nb)) || (rc = validate_tensor("o", o, true, nb)))
         return rc;
     if (!lse || !g) return fail(FOCUS_ERR_INVALID_ARG, "lse or g is NULL");
     if ((uintptr_t)g % 16) return fail(FOCUS_ERR_INVALID_ARG, "g is not 16-byte aligned");

@@ -18,8 +18,9 @@ int check_cuda(cudaError_t e, const char* what);
 
 // shape validation shared by all entry points (0 or a negative status)
 int validate_shape(const focus_shape* s);
-// validation of a bf16 tensor argument; tma = also enforce 16-byte base alignment and stride % 8 == 0
-int validate_tensor(const char* name, const focus_tensor& t, bool tma);
+// validation of a bf16 tensor argument; tma = also enforce 16-byte base alignment and stride % 8 == 0;
+// batch > 1 requires a positive batch stride
+int validate_tensor(const char* name, const focus_tensor& t, bool tma, int batch);
 // current device must be compute capability 10.x
 int require_sm100();
 
@@ -80,7 +81,6 @@ struct AttnArgs {
     int gate_ld = 0;
     float gate_lambda = 0.f;
 };
-int launch_attn_simple(const AttnArgs& a, cudaStream_t st);
 int launch_attn_sm100(const AttnArgs& a, cudaStream_t st);
 
 }  // namespace focus

@@ -16,7 +16,9 @@ constexpr int MAX_DEVICES = 64;
 static uint32_t* g_scratch_addr[MAX_DEVICES];
 static std::mutex g_scratch_mutex;
 
-// Device address of the scratch array on the current device; looked up once per device.
+// Device address of the scratch array on the current device; looked up once per device and kept for
+// the life of the process.  An application that destroys the device's primary context
+// (cudaDeviceReset) invalidates the address: this entry point must not be used after that.
 static int scratch_address(uint32_t** out) {
     int dev = 0;
     int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
@@ -100,6 +102,9 @@ extern "C" int focus_count_kept_noalloc(const focus_shape* shape, const uint32_t
                     "focus_count_kept_noalloc needs %zu bytes of scratch (batch*Hkv*ceil(n/128)*K*16) but the built-in "
                     "array holds %d; use focus_count_kept with a caller-allocated workspace", need,
                     (int)FOCUS_NOALLOC_MAX_BYTES);
+    // heads are the second grid dimension of both kernels: refuse before anything is enqueued
+    if (HQ > 65535 || HK > 65535)
+        return fail(FOCUS_ERR_UNSUPPORTED, "focus_count_kept_noalloc: batch*Hq (%d) and batch*Hkv (%d) must not exceed 65535", HQ, HK);
     if ((rc = require_sm100())) return rc;
     uint32_t* scratch = nullptr;
     if ((rc = scratch_address(&scratch))) return rc;

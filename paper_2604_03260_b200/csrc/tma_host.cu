@@ -36,7 +36,7 @@ int make_tmap_bf16_4d(CUtensorMap* out, const void* base, uint64_t d0, uint64_t 
 int make_tmap_qkv(CUtensorMap* out, const focus_tensor& t, int batch, int H, int n, int D, int rows) {
     // a dimension of extent 1 still needs a legal (multiple of 16 bytes, non-zero) stride
     uint64_t sb = (uint64_t)t.stride_b * 2;
-    if (batch == 1 || sb == 0) sb = (uint64_t)t.stride_h * 2 * (uint64_t)H;
+    if (batch == 1) sb = (uint64_t)t.stride_h * 2 * (uint64_t)H;
     return make_tmap_bf16_4d(out, t.ptr, (uint64_t)D, (uint64_t)n, (uint64_t)H, (uint64_t)batch,
                              (uint64_t)t.stride_n * 2, (uint64_t)t.stride_h * 2, sb, 64, (uint32_t)rows);
 }

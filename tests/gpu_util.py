@@ -45,6 +45,20 @@ def as_u32(t):
     return t.detach().cpu().numpy().view(np.uint32)
 
 
+def masks_vs_oracle(wl, X, C, masks):
+    """membership masks of the CUDA path against oracle.assign on the same bits: bit-exact except where the
+    fp64 margin between the last group taken and the first one left is below 1e-5 (near-ties, counted).
+    Returns (mismatches inside near-ties, near-ties)."""
+    ref, margins = fo.assign(fi.bf16_bits(X), C.cpu().numpy(), wl.topk)
+    got = as_u32(masks)
+    bad = got != ref
+    near = margins < 1e-5
+    outside = bad & ~near
+    assert not outside.any(), (f"{int(outside.sum())} masks differ from the oracle outside near-ties, first at "
+                               f"(head, token) {np.argwhere(outside)[0].tolist()}")
+    return int(bad.sum()), int(near.sum())
+
+
 def compare_rows(wl, Q, K, V, mq_np, mk_np, O, lse, rows=None, dense=False):
     """oracle on the given rows (all rows when None) vs the GPU outputs; returns error statistics"""
     qb, kb, vb = fi.bf16_bits(Q), fi.bf16_bits(K), fi.bf16_bits(V)

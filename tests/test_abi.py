@@ -141,3 +141,52 @@ def test_training_forward_host_checks():
     assert L.focus_gate_attn_fwd(ctypes.byref(capped), t_ok, t_ok, t_ok, 4096, 5.0, t_ok, 4096, None, None) == -2   # unsupported
     many = fb.make_shape(8, 2, 1000, 128, 16, 2, 64)
     assert L.focus_gate_attn_fwd(ctypes.byref(many), t_ok, t_ok, t_ok, 4096, 5.0, t_ok, 4096, None, None) == -2
+
+
+def test_tensor_arguments_that_would_alias_or_misalign_are_refused():
+    """batch > 1 with a zero batch stride, and decode query vectors that cannot be read two elements at a time"""
+    L = fb.lib()
+    s2 = fb.make_shape(8, 4, 1000, 128, 4, 2, 16, batch=2)
+    t_ok = fb.focus_tensor(4096, 8 * 1000 * 128, 1000 * 128, 128)
+    t_b0 = fb.focus_tensor(4096, 0, 1000 * 128, 128)
+    assert L.focus_attn_fwd(ctypes.byref(s2), t_b0, t_ok, t_ok, None, None, None, 0, t_ok, 4096, None, None) == -1
+    assert b"stride_b" in L.focus_last_error()
+    assert L.focus_attn_fwd(ctypes.byref(s2), t_ok, t_ok, t_b0, None, None, None, 0, t_ok, 4096, None, None) == -1
+    assert L.focus_assign(ctypes.byref(s2), t_b0, 8, 4096, 4096, None, 1e-5, None) == -1
+    s1 = fb.make_shape(8, 4, 1000, 128, 4, 2, 16)
+    kv = fb.focus_tensor(4096, 4 * 1000 * 128, 1000 * 128, 128)
+    vec = lambda ptr, sb, sh: fb.focus_tensor(ptr, sb, sh, 128)
+    big = 1 << 30
+    for bad_q in (vec(4098, 8 * 128, 128), vec(4096, 8 * 128, 129), vec(4096, 8 * 128 + 1, 128)):
+        assert L.focus_decode_step(ctypes.byref(s1), bad_q, kv, kv, 4096, 4096, vec(4096, 8 * 128, 128), 4096, 4096, big, None) == -1
+    assert L.focus_decode_step(ctypes.byref(s2), vec(4096, 0, 128), kv, kv, 4096, 4096, vec(4096, 8 * 128, 128), 4096, 4096, big, None) == -1
+    # the no-allocation count: too many heads for its launch shape is refused before anything is enqueued
+    wide = fb.make_shape(70000, 1, 1, 64, 1, 1, 0)
+    assert L.focus_count_kept_noalloc(ctypes.byref(wide), 4096, 4096, 4096, None) == -2
+
+
+def test_ctypes_structs_match_the_header(tmp_path):
+    """sizeof / offsetof of the three ABI structs as a C compiler sees them in include/focus.h"""
+    import subprocess
+    structs = {"focus_shape": fb.focus_shape, "focus_tensor": fb.focus_tensor, "focus_tiles_layout": fb.focus_tiles_layout}
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "focus.h"', 'int main(void) {']
+    for name, cls in structs.items():
+        lines.append(f'  printf("{name} %zu\\n", sizeof({name}));')
+        for field, _ in cls._fields_:
+            lines.append(f'  printf("{name}.{field} %zu\\n", offsetof({name}, {field}));')
+    lines += ['  return 0;', '}']
+    src = tmp_path / "abi_probe.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "abi_probe"
+    subprocess.check_call(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)])
+    seen = dict(l.split() for l in subprocess.check_output([str(exe)], text=True).splitlines())
+    for name, cls in structs.items():
+        assert int(seen[name]) == ctypes.sizeof(cls), name
+        for field, _ in cls._fields_:
+            assert int(seen[f"{name}.{field}"]) == getattr(cls, field).offset, (name, field)
+    # and the header has no field the binding lacks
+    text = open(os.path.join(ROOT, "include", "focus.h")).read()
+    body = re.search(r"typedef struct \{([^}]*)\} focus_tiles_layout;", text, re.S).group(1)
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    declared = [n.strip() for decl in body.split(";") if decl.strip() for n in decl.strip().split(None, 1)[1].split(",")]
+    assert declared == [f for f, _ in fb.focus_tiles_layout._fields_]

@@ -44,6 +44,20 @@ def test_assign_shapes(D, K, t, n):
     check(wl, Kt, C.contiguous(), wl.Hkv)
 
 
+@pytest.mark.parametrize("name", ["cfg3", "cfg4", "M128k", "cfg5"])
+def test_assign_large_configs_at_full_size(name):
+    """every mask of the large configurations (clustered K = 8 at 32K, D = 256 top-1 at 64K, the 128K metric point,
+    and 1M tokens, where element offsets pass 2^32) against the oracle; near-ties counted and reported"""
+    wl = fi.WORKLOADS[name]
+    Q, K, V, C = fi.make_inputs(wl, "cuda")
+    del V
+    diff_k, near_k = check(wl, K, C, wl.Hkv)
+    diff_q, near_q = check(wl, Q, C, wl.Hq)
+    print(f"{wl.name}: near-ties Q {near_q} K {near_k} of {(wl.Hq + wl.Hkv) * wl.n} vectors; "
+          f"masks differing inside near-ties Q {diff_q} K {diff_k}")
+    assert near_q + near_k < 1e-4 * (wl.Hq + wl.Hkv) * wl.n + 16
+
+
 def test_assign_clustered_and_ties():
     wl = fi.WORKLOADS["cfg3"].with_n(4096)
     Q, K, V, C = fi.make_inputs(wl, "cuda")

@@ -68,22 +68,3 @@ def test_feeds_the_attention_path():
         ws, _ = gpu_tiles(wl, mq, mk, layout)
         O, lse = gpu_attn(wl, Q, K, V, mq, mk, ws, layout)
         assert_parity(compare_rows(wl, Q, K, V, as_u32(mq), as_u32(mk), O, lse))
-
-
-def test_throughput_is_reported():
-    """Llama-3-8B-shaped hidden states (d_model 4096, d_g 16, K 4) at 128K tokens: time and GB/s, printed for the log"""
-    n, d = 131072, 4096
-    h, Wg, C, bias = hidden_inputs(n, d, 16, 4, 3)
-    shape = fb.make_shape(32, 8, n, 128, 4, 2, 2048)
-    folded = torch.empty((4, d), dtype=torch.float32, device="cuda")
-    mq = torch.empty((32, n), dtype=torch.int32, device="cuda"); mk = torch.empty((8, n), dtype=torch.int32, device="cuda")
-    ts = []
-    for i in range(5):
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(); fb.focus_assign_hidden(shape, h, Wg, C, bias, folded, mq, mk); b.record()
-        torch.cuda.synchronize()
-        ts.append(a.elapsed_time(b))
-    ms = float(np.median(ts[1:]))
-    gbs = (n * d * 2 + 40 * n * 4) / ms / 1e6
-    print(f"focus_assign_hidden 128K x 4096: {ms:.3f} ms, {gbs:.0f} GB/s")
-    assert gbs > 500

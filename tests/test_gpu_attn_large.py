@@ -6,7 +6,7 @@ import torch
 
 from paper_2604_03260_b200 import binding as fb
 from paper_2604_03260_b200 import inputs as fi
-from tests.gpu_util import as_u32, assert_parity, compare_rows, gpu_assign, gpu_attn, gpu_tiles
+from tests.gpu_util import as_u32, assert_parity, compare_rows, gpu_assign, gpu_attn, gpu_tiles, masks_vs_oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -16,6 +16,9 @@ def run_sampled(name, per_head, layout=0, dense_too=False):
     Q, K, V, C = fi.make_inputs(wl, "cuda")
     mq, _ = gpu_assign(wl, Q, C, wl.Hq)
     mk, _ = gpu_assign(wl, K, C, wl.Hkv)
+    # the masks both sides use below are the oracle's own except at counted near-ties
+    masks_vs_oracle(wl, Q, C, mq)
+    masks_vs_oracle(wl, K, C, mk)
     ws, L = gpu_tiles(wl, mq, mk, layout)
     O, lse = gpu_attn(wl, Q, K, V, mq, mk, ws, layout)
     rows = fi.sample_rows(wl, per_head)

@@ -77,34 +77,3 @@ def test_decode_argument_checks():
     with pytest.raises(fb.FocusError) as e:        # workspace too small
         fb.focus_decode_step(shape, Q[:4, -1].contiguous(), K, V, m[:4, 0].contiguous(), m[:2], o[:4], lse[:4], ws[:16])
     assert e.value.status == -3
-
-
-def test_decode_throughput_is_reported():
-    """128K cached tokens, Llama-3-8B-shaped layer: time per step and bytes of attended K/V rows per second"""
-    wl = fi.WORKLOADS["M128k"]
-    Q, K, V, C = fi.make_inputs(wl, "cuda")
-    shape = fb.shape_of(wl)
-    mq = torch.empty((wl.Hq, wl.n), dtype=torch.int32, device="cuda"); mk = torch.empty((wl.Hkv, wl.n), dtype=torch.int32, device="cuda")
-    fb.focus_assign(shape, Q, wl.Hq, C, mq); fb.focus_assign(shape, K, wl.Hkv, C, mk)
-    q_new = Q[:, -1].contiguous(); mq_new = mq[:, -1].contiguous()
-    o = torch.empty((wl.Hq, wl.D), dtype=torch.bfloat16, device="cuda"); lse = torch.empty(wl.Hq, device="cuda")
-    ws = torch.empty(fb.focus_decode_workspace_bytes(shape), dtype=torch.uint8, device="cuda")
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    ts = []
-    for i in range(6):
-        flush.zero_()                                            # K/V (512 MB) exceed L2, the flush makes it explicit
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(); fb.focus_decode_step(shape, q_new, K, V, mq_new, mk, o, lse, ws); b.record()
-        torch.cuda.synchronize()
-        ts.append(a.elapsed_time(b))
-    ms = float(np.median(ts[1:]))
-    # a key row is read when any of the 4 query heads of its KV head attends it
-    mqn = mq_new.cpu().numpy().view(np.uint32).reshape(wl.Hkv, wl.G); mkn = mk.cpu().numpy().view(np.uint32)
-    rows = 0
-    for hk in range(wl.Hkv):
-        union = np.bitwise_or.reduce(mqn[hk])
-        far = (mkn[hk, : wl.n - 1 - wl.window] & union) != 0
-        rows += int(far.sum()) + wl.window + 1
-    gbs = rows * 2 * wl.D * 2 / ms / 1e6
-    print(f"focus_decode_step at 128K cached tokens: {ms:.3f} ms, {rows} of {wl.Hkv * wl.n} K/V row pairs read, {gbs:.0f} GB/s")
-    assert gbs > 300

@@ -453,7 +453,8 @@ def test_bias_is_the_inference_residue_of_sinkhorn_column_scaling():
     assert (plain != want).any()            # without the bias the unbalanced ranking differs
     mass = Q.sum(axis=0)                     # Sinkhorn did balance the groups' mass; the plain row softmax does not
     P = np.exp(S / tau); P /= P.sum(axis=1, keepdims=True)
-    assert mass.max() / mass.min() < 0.5 * P.sum(axis=0).max() / P.sum(axis=0).min()
+    # (Sinkhorn converges linearly: ten iterations leave these inputs within 5 % of balance, the row softmax is 2x off)
+    assert mass.max() / mass.min() < 1.05 < 2.0 < P.sum(axis=0).max() / P.sum(axis=0).min()
 
 
 # ---------------------------------------------------------------- training-time forward: Sinkhorn and the soft gate (Sec. 2)

@@ -7,6 +7,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import focus_oracle as fo
 from paper_2604_03260_b200 import binding as fb
 from paper_2604_03260_b200 import inputs as fi
 
@@ -50,6 +51,9 @@ def test_two_calls_in_a_row_match_the_workspace_variant():
     got = without_allocation(shape2, mq2, mk2)
     assert torch.equal(got, with_workspace(shape2, mq2, mk2))
     assert (got > 0).all()
+    # the count is the size of the attended set as the CPU oracle counts it from the mask definition
+    want = fo.kept_pairs(mq2.cpu().numpy().view(np.uint32), mk2.cpu().numpy().view(np.uint32), small.window)
+    assert np.array_equal(got.numpy(), want)
     # and the first problem again gives the first answer again
     assert torch.equal(without_allocation(shape, mq, mk), with_workspace(shape, mq, mk))
 
