@@ -335,6 +335,16 @@ FOCUS_API int focus_gate_attn_fwd(const focus_shape* shape, focus_tensor q, focu
 FOCUS_API int focus_selftest_umma(int32_t D, const void* a, const void* b, const void* p, const void* v, float* s_out,
                         float* o_out, int32_t* dev_status, void* stream);
 
+/*
+ * focus_selftest_umma_pair -- diagnostic (the paper has no counterpart): the same two tiles with D = 128 through one
+ * MMA shared by a pair of CTAs on neighbouring SMs, the form focus_attn_fwd uses at D = 128: 256 rows of A and P (128
+ * per CTA), each CTA staging half of B (64 of its 128 rows) and half of V (64 of its 128 columns).
+ *   a, p      device bf16 [256, 128] row-major     b, v   device bf16 [128, 128] row-major
+ *   s_out, o_out   device fp32 [256, 128]          dev_status   as above
+ */
+FOCUS_API int focus_selftest_umma_pair(const void* a, const void* b, const void* p, const void* v, float* s_out,
+                                       float* o_out, int32_t* dev_status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

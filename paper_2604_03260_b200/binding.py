@@ -99,6 +99,8 @@ def lib():
         L.focus_count_kept_noalloc.argtypes = [SP, vp, vp, vp, vp]
         L.focus_selftest_umma.restype = C.c_int
         L.focus_selftest_umma.argtypes = [i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.focus_selftest_umma_pair.restype = C.c_int
+        L.focus_selftest_umma_pair.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -229,6 +231,10 @@ def focus_count_kept_noalloc(shape, mq, mk, counts_out, stream=None):
 def focus_selftest_umma(D, a, b, p, v, s_out, o_out, dev_status, stream=None):
     _check(lib().focus_selftest_umma(D, _p(a), _p(b), _p(p), _p(v), _p(s_out), _p(o_out), _p(dev_status),
                                      _stream(stream)))
+
+
+def focus_selftest_umma_pair(a, b, p, v, s_out, o_out, dev_status, stream=None):
+    _check(lib().focus_selftest_umma_pair(_p(a), _p(b), _p(p), _p(v), _p(s_out), _p(o_out), _p(dev_status), _stream(stream)))
 
 
 def alloc_workspace(shape, layout, device="cuda") -> torch.Tensor:
