@@ -84,6 +84,8 @@ struct AttnParams {
     int gate_ld;
     float gate_hl;
     // window pass of the split layout: only the tiles that reach into the window, only pairs WITHOUT a shared group
+    // class-sorted pass of the split layout: only pairs WITH a shared group (the window pass covers the others)
+    int share_only;
     int local_only;
     float* o32;              // partial passes: O in fp32, rows [B*Hq][n][D], instead of bf16 to `o`
 };
@@ -98,18 +100,15 @@ struct TileWalk {
     bool far_phase;
     // class-sorted layout: the ranges of sorted key tiles, key class by key class
     const int32_t* qr;
-    const int32_t* qr2;         // CTA pair: the ranges of the second block of 256 sorted queries (or nullptr)
     int nck, jk, rend;
     bool sorted;
 
-    // a0 = first 128-row query tile of the item, nq = number of query tiles of the item: 1 or 2 for one CTA, 4 for a
-    // CTA pair (two blocks of 256 queries, one per CTA, which walk the union of their key tiles together)
+    // a0 = first 128-row query tile of the item, nq = number of query tiles of the item (1 or 2)
     __device__ __forceinline__ void init(const AttnParams& p, int hq, int a0, int nq) {
         sorted = p.sorted != 0;
         if (sorted) {
             const int hk = (hq / p.Hq) * p.Hkv + (hq % p.Hq) / p.G;
             qr = p.qrange + ((size_t)hq * p.nqblk + (a0 >> 1)) * FOCUS_MAX_CLASSES * 2;
-            qr2 = (nq == 4 && (a0 >> 1) + 1 < p.nqblk) ? qr + FOCUS_MAX_CLASSES * 2 : nullptr;
             nck = __ldg(p.ncls_k + hk);
             jk = -1;
             b = rend = 0;
@@ -139,13 +138,6 @@ struct TileWalk {
                 if (++jk >= nck) return -1;
                 b = __ldg(qr + 2 * jk);
                 rend = __ldg(qr + 2 * jk + 1);
-                if (qr2) {          // union with the other block's range of this class (an empty range has first = last)
-                    const int b2 = __ldg(qr2 + 2 * jk), e2 = __ldg(qr2 + 2 * jk + 1);
-                    if (e2 > b2) {
-                        if (rend > b) { b = min(b, b2); rend = max(rend, e2); }
-                        else { b = b2; rend = e2; }
-                    }
-                }
             }
             return b++;
         }
@@ -267,16 +259,20 @@ __device__ __forceinline__ int count_le_128(const int32_t* __restrict__ a, int v
 // position and, unless the classes share a group, not further back than the window.  The decisions
 // "no mask needed" / "nothing attended" are taken per warp from the warp's smallest and largest row
 // position.
+// `window_ok` = false (class-sorted pass of the split layout): a row that shares no group with the tile's class keeps
+// nothing of it, whatever the distance.
 __device__ __forceinline__ void build_tile_mask_sorted(TileMask& tm, int w, const int32_t* __restrict__ kpos, bool share,
-                                                       int pos, int wmin, int wmax) {
+                                                       int pos, int wmin, int wmax, bool window_ok) {
     const int k_first = __ldg(kpos), k_last = __ldg(kpos + 127);
     tm.all_masked = wmax < 0 || k_first > wmax;
+    const bool none = !share && !window_ok;
+    const bool any_none = __any_sync(0xffffffffu, none);        // (every lane takes part: no short-circuit before it)
     const bool need_causal = k_last > wmin;
     const bool need_window = !share && ((long long)wmax - k_first > w);
-    tm.masked = need_causal || need_window;
+    tm.masked = need_causal || need_window || any_none;
     tm.kw[0] = tm.kw[1] = tm.kw[2] = tm.kw[3] = 0xffffffffu;
     if (tm.masked && !tm.all_masked) {
-        const int hi = need_causal ? (pos < 0 ? 0 : count_le_128(kpos, pos)) : 128;          // columns < hi are causal
+        const int hi = none ? 0 : (need_causal ? (pos < 0 ? 0 : count_le_128(kpos, pos)) : 128);          // columns < hi are causal
         const long long edge = (long long)pos - w - 1;
         const int lo = (need_window && pos >= 0 && edge >= 0) ? count_le_128(kpos, (int)edge) : 0;   // columns >= lo are in the window
 #pragma unroll

@@ -447,7 +447,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (p.sorted) {
                     const bool share = (mi & __ldg(p.cls_k + (size_t)hk * FOCUS_MAX_CLASSES + walk.jk)) != 0u;
                     build_tile_mask_sorted(tm, p.w, p.perm_k + (size_t)hk * p.nkp + (size_t)kb * 128, share,
-                                           valid ? (int)i : -1, wmin, wmax);
+                                           valid ? (int)i : -1, wmin, wmax, !p.share_only);
                 } else {
                     build_tile_mask(tm, p, a, kb, i, mi, aq, f_x, hk);
                 }
@@ -737,6 +737,7 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
     p.counters = a.ws ? reinterpret_cast<const unsigned long long*>(a.ws + a.L.counters) : nullptr;
     p.gate_g = a.gate_g; p.gate_ld = a.gate_ld; p.gate_hl = 0.5f * a.gate_lambda;
     p.local_only = a.local_pass ? 1 : 0;
+    p.share_only = (sorted && a.L.layout == FOCUS_LAYOUT_SORTED_LOCAL) ? 1 : 0;
     p.o32 = a.o32;
     if (sorted) p.nitems = (long long)a.s.batch * a.s.Hq * p.nqblk * p.ipb;
     int dev = 0, sms = 0;
