@@ -217,7 +217,9 @@ FOCUS_API int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, co
  *   lse         device fp32 [batch*Hq, n], natural log
  *   dev_status  device int32[4], nullable: [0] stays 0 on success.  [0] = 1: a bounded wait inside the
  *               kernel expired (the kernel then drains and exits; outputs are invalid), [1] = code of
- *               the wait, [2] = work item, [3] = CTA.  [0] = 2: a class-sorted layout was asked for
+ *               the wait (10, 11: the load role waiting for a free query buffer / ring slot; 20-26: the
+ *               MMA role waiting for queries, a ring stage or probabilities; 30-41: a softmax role
+ *               waiting for S, its partner thread or O), [2] = work item, [3] = CTA.  [0] = 2: a class-sorted layout was asked for
  *               but a head holds more than FOCUS_MAX_CLASSES distinct mask values (possible only with
  *               masks that do not come from a top-k rule); nothing was computed and O / lse were not
  *               written.  Pass a non-NULL dev_status with layouts 1 and 3 when the masks are not the
@@ -334,6 +336,21 @@ FOCUS_API int focus_gate_attn_fwd(const focus_shape* shape, focus_tensor q, focu
  */
 FOCUS_API int focus_selftest_umma(int32_t D, const void* a, const void* b, const void* p, const void* v, float* s_out,
                         float* o_out, int32_t* dev_status, void* stream);
+
+/*
+ * focus_selftest_stalled_wait -- diagnostic (the paper has no counterpart): runs the attention kernel in dense causal
+ * mode with one stage of its K/V ring deliberately left unfilled, so that the role waiting for that stage runs into
+ * its time limit.  Every wait inside the attention kernels is bounded (4 s in focus_attn_fwd); this entry point sets
+ * the bound to `wait_limit_ns` and shows the exit taken when it expires: dev_status[0] = 1, [1] = code of the wait
+ * that gave up, [2] = work item, [3] = CTA; the other roles of the CTA notice, nothing traps or hangs, tensor memory
+ * is released and the kernel returns.  O and lse are left incomplete.  The device and the context stay usable.
+ *   shape, q, k, v, o, lse   as for focus_attn_fwd (n >= 512; masks are not used)
+ *   wait_limit_ns            1000 ... 4000000000; the bound is checked at a granularity of about 0.1 s
+ *   dev_status               device int32[4], zeroed by the caller, required
+ */
+FOCUS_API int focus_selftest_stalled_wait(const focus_shape* shape, focus_tensor q, focus_tensor k, focus_tensor v,
+                                          focus_tensor o, float* lse, unsigned long long wait_limit_ns,
+                                          int32_t* dev_status, void* stream);
 
 /*
  * focus_selftest_umma_pair -- diagnostic (the paper has no counterpart): the same two tiles with D = 128 through one

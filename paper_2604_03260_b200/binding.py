@@ -101,6 +101,8 @@ def lib():
         L.focus_selftest_umma.argtypes = [i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.focus_selftest_umma_pair.restype = C.c_int
         L.focus_selftest_umma_pair.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+        L.focus_selftest_stalled_wait.restype = C.c_int
+        L.focus_selftest_stalled_wait.argtypes = [SP, focus_tensor, focus_tensor, focus_tensor, focus_tensor, vp, C.c_uint64, vp, vp]
         _lib = L
     return _lib
 
@@ -235,6 +237,11 @@ def focus_selftest_umma(D, a, b, p, v, s_out, o_out, dev_status, stream=None):
 
 def focus_selftest_umma_pair(a, b, p, v, s_out, o_out, dev_status, stream=None):
     _check(lib().focus_selftest_umma_pair(_p(a), _p(b), _p(p), _p(v), _p(s_out), _p(o_out), _p(dev_status), _stream(stream)))
+
+
+def focus_selftest_stalled_wait(shape, q, k, v, o, lse, wait_limit_ns, dev_status, stream=None):
+    _check(lib().focus_selftest_stalled_wait(C.byref(shape), tensor_arg(q), tensor_arg(k), tensor_arg(v), tensor_arg(o), _p(lse),
+                                             wait_limit_ns, _p(dev_status), _stream(stream)))
 
 
 def alloc_workspace(shape, layout, device="cuda") -> torch.Tensor:

@@ -337,6 +337,33 @@ int focus_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k, foc
     return launch_attn_sm100(a, (cudaStream_t)stream);
 }
 
+int focus_selftest_stalled_wait(const focus_shape* shape, focus_tensor q, focus_tensor k, focus_tensor v, focus_tensor o,
+                                float* lse, unsigned long long wait_limit_ns, int32_t* dev_status, void* stream) {
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    const int nb = shape->batch;
+    if ((rc = validate_tensor("q", q, true, nb)) || (rc = validate_tensor("k", k, true, nb)) ||
+        (rc = validate_tensor("v", v, true, nb)) || (rc = validate_tensor("o", o, true, nb)))
+        return rc;
+    if (!lse || !dev_status) return fail(FOCUS_ERR_INVALID_ARG, "lse or dev_status is NULL");
+    if (wait_limit_ns < 1000ull || wait_limit_ns > 4000000000ull)
+        return fail(FOCUS_ERR_INVALID_ARG, "wait_limit_ns must lie between 1 microsecond and 4 seconds");
+    if (shape->n < 512) return fail(FOCUS_ERR_INVALID_ARG, "n must be at least 512 (the stalled stage is the fourth of an item)");
+    if ((rc = require_sm100())) return rc;
+    AttnArgs a;
+    a.s = *shape;
+    a.q = q; a.k = k; a.v = v; a.o = o;
+    a.mq = nullptr; a.mk = nullptr;
+    a.ws = nullptr;                        // dense causal walk
+    a.lse = lse;
+    a.dev_status = dev_status;
+    a.scale = shape->scale > 0.f ? shape->scale : 1.0f / sqrtf((float)shape->D);
+    memset(&a.L, 0, sizeof a.L);
+    a.wait_limit_ns = wait_limit_ns;
+    a.stall_at = 3;
+    return launch_attn_sm100(a, (cudaStream_t)stream);
+}
+
 int focus_gate_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k, focus_tensor v, const float* g, float lambda,
                         focus_tensor o, float* lse, int32_t* dev_status, void* stream) {
     int rc = validate_shape(shape);

@@ -88,6 +88,8 @@ struct AttnParams {
     int share_only;
     int local_only;
     float* o32;              // partial passes: O in fp32, rows [B*Hq][n][D], instead of bf16 to `o`
+    unsigned long long wait_limit_ns;   // bound of every wait inside the kernel
+    long long stall_at;      // diagnostic: index of a K/V ring stage the producer leaves unfilled (-1 = none)
 };
 
 // Enumerates the key tiles a 256-row query block visits, in increasing order.  Every role of the

@@ -67,6 +67,7 @@ struct SharedCtl {
     uint64_t xchg[4];                 // split rows, per 32-row quadrant: both column halves have published a per-row value
     uint64_t gbar[2];                 // soft gate, per softmax warpgroup: the key assignments of the tile are in shared memory
     uint64_t kv_full[8], kv_empty[8];
+    unsigned long long limit_ns;      // how long a wait may last before the role gives up
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -81,7 +82,7 @@ __device__ __forceinline__ bool ctl_wait(uint64_t* bar, uint32_t parity, SharedC
         for (int it = 0; it < 128; ++it)
             if (mbar_try_wait(a, parity)) return true;
         if (*(volatile int*)&ctl->abort_flag) return false;
-        if (globaltimer_ns() - t0 > 4000000000ull) return false;
+        if (globaltimer_ns() - t0 > ctl->limit_ns) return false;
     }
 }
 
@@ -134,6 +135,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             mbar_init(smem_u32(&ctl.kv_empty[s]), 1);
         }
         ctl.abort_flag = 0;
+        ctl.limit_ns = p.wait_limit_ns;
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -173,6 +175,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 // one K or V tile into the next stage(s) of the ring
                 auto load_tile = [&](bool is_v, int tile) {
                     for (int part = 0; part < C::PARTS; ++part) {
+                        if (nload == p.stall_at) { ++nload; continue; }      // diagnostic: this stage is never filled
                         const int slot = (int)(nload % C::NSTAGE);
                         const long long use = nload / C::NSTAGE;
                         if (use > 0 && !ctl_wait(&ctl.kv_empty[slot], (uint32_t)((use - 1) & 1), &ctl)) {
@@ -681,6 +684,11 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // ---------------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
+    if (*(volatile int*)&ctl.abort_flag) {
+        // a role gave up: let copies that were already issued land before the CTA leaves
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 20000ull) { }
+    }
     if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
@@ -739,6 +747,8 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
     p.local_only = a.local_pass ? 1 : 0;
     p.share_only = (sorted && a.L.layout == FOCUS_LAYOUT_SORTED_LOCAL) ? 1 : 0;
     p.o32 = a.o32;
+    p.wait_limit_ns = a.wait_limit_ns;
+    p.stall_at = a.stall_at;
     if (sorted) p.nitems = (long long)a.s.batch * a.s.Hq * p.nqblk * p.ipb;
     int dev = 0, sms = 0;
     if ((rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice"))) return rc;

@@ -80,6 +80,8 @@ struct AttnArgs {
     const float* gate_g = nullptr;   // training-time soft gate: assignments [batch, n, gate_ld]; nullptr = no gate
     int gate_ld = 0;
     float gate_lambda = 0.f;
+    unsigned long long wait_limit_ns = 4000000000ull;   // every wait inside the kernel gives up after this long
+    long long stall_at = -1;         // diagnostic (focus_selftest_stalled_wait): a ring stage that is never filled
 };
 int launch_attn_sm100(const AttnArgs& a, cudaStream_t st);
 

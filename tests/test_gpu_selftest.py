@@ -3,6 +3,7 @@ import pytest
 import torch
 
 from paper_2604_03260_b200 import binding as fb
+from paper_2604_03260_b200 import inputs as fi
 
 pytestmark = pytest.mark.gpu
 
@@ -42,3 +43,27 @@ def test_umma_tiles_shared_by_a_cta_pair_match_matmul():
     o_ref = p.double() @ v.double()
     assert (s.double() - s_ref).abs().max().item() < 1e-3 * max(1.0, s_ref.abs().max().item())
     assert (o.double() - o_ref).abs().max().item() < 1e-3 * max(1.0, o_ref.abs().max().item())
+
+
+@pytest.mark.parametrize("D", [64, 128, 256])
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(D):
+    """one stage of the K/V ring is never filled: the waiting role gives up after its limit, the kernel says where,
+    releases tensor memory and returns; the next ordinary launch in the same process is correct"""
+    from tests.gpu_util import assert_parity, compare_rows, gpu_attn
+    import numpy as np
+    wl = fi.Workload("stall", 2, 1, D, 1500, 4, 2, 8, seed=40 + D)
+    Q, K, V, C = fi.make_inputs(wl, "cuda")
+    shape = fb.shape_of(wl)
+    O = torch.zeros_like(Q)
+    lse = torch.zeros((wl.Hq, wl.n), dtype=torch.float32, device="cuda")
+    st = torch.zeros(4, dtype=torch.int32, device="cuda")
+    fb.focus_selftest_stalled_wait(shape, Q, K, V, O, lse, 2_000_000, st)
+    torch.cuda.synchronize()                       # returns: nothing hangs, nothing faults
+    code = st.cpu().tolist()
+    # whichever role started waiting first reports: the MMA role for the stage itself (21-23), the producer for the ring
+    # slot that is never handed back (10, 11), or a softmax role for the S / O that never comes (30, 31, 40, 41)
+    assert code[0] == 1 and code[1] in (10, 11, 21, 22, 23, 30, 31, 40, 41), code
+    assert 0 <= code[3] < 148
+    masks = np.full((wl.Hq, wl.n), 0b11, np.uint32), np.full((wl.Hkv, wl.n), 0b11, np.uint32)
+    O2, lse2 = gpu_attn(wl, Q, K, V)                # asserts a clean status itself
+    assert_parity(compare_rows(wl, Q, K, V, masks[0], masks[1], O2, lse2, dense=True))
