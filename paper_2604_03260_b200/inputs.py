@@ -9,6 +9,12 @@ these draws stand in for them:
 * centroids: fp32 N(0,1) rows of shape [Hkv, K, D], each normalised to unit length.
 * ``clustered`` workloads: one latent label z_i per token from a skewed categorical; every query
   head vector and every key head vector of token i is 2.0 * c[kv(h), z_i] + N(0, I); V stays N(0,1).
+* ``runs`` workloads (memberships coherent over positions, as a trained router gives for text whose
+  topic persists): the sequence is cut into runs of geometric length (mean ``runs`` tokens); a run draws
+  ``topk`` distinct latent groups, a token keeps its run's groups except with probability ``flip``
+  (then it draws its own); every query and key head vector of the token is
+  ``signal`` * (sum of the centroids of its latent groups) + N(0, I).  Whole 128-token tiles then
+  hold one set of groups, so far tiles die or need no mask at all.
 
 Draw order with one ``torch.Generator`` seeded by ``Workload.seed``: centroids, (z), then per head
 Q rows, per KV head K rows, per KV head V rows.
@@ -35,6 +41,9 @@ class Workload:
     scale: float = 0.0          # 0 -> 1/sqrt(D)
     clustered: bool = False
     seed: int = 0
+    runs: float = 0.0           # > 0: run-structured latent groups, mean run length in tokens
+    flip: float = 0.0           # probability that a token leaves its run's groups
+    signal: float = 5.0         # amplitude of the latent centroids in a run-structured draw
 
     @property
     def G(self) -> int:
@@ -61,6 +70,9 @@ WORKLOADS = {
     "cfg4": Workload("cfg4-gemma2-9b-softcap", 16, 8, 256, 65536, 4, 1, 4096, softcap=50.0, seed=1004),
     "cfg5": Workload("cfg5-llama3-8b-1m", 32, 8, 128, 1048576, 4, 2, 2048, seed=1005),
     "M128k": Workload("M-llama3-8b-128k", 32, 8, 128, 131072, 4, 2, 2048, seed=1006),
+    # the metric point's shape with memberships coherent over positions (runs of ~512 tokens, 0.1 % stray tokens)
+    "Mruns": Workload("M-llama3-8b-128k-runs", 32, 8, 128, 131072, 4, 2, 2048, seed=1007, runs=512.0, flip=0.001),
+    "Mruns1": Workload("M-llama3-8b-128k-runs-top1", 32, 8, 128, 131072, 4, 1, 2048, seed=1008, runs=512.0, flip=0.001),
 }
 
 
@@ -82,19 +94,33 @@ def make_inputs(wl: Workload, device: str = "cpu"):
     C = torch.randn((wl.Hkv, wl.K, wl.D), generator=gen, device=device, dtype=torch.float32)
     C = C / C.norm(dim=-1, keepdim=True)
     z = None
+    member = None               # runs: [n, K] 0/1 latent memberships
     if wl.clustered:
         p = torch.tensor(SKEW[: wl.K], dtype=torch.float32, device=device)
         p = p / p.sum()
         z = torch.multinomial(p, wl.n, replacement=True, generator=gen)
+    elif wl.runs > 0:
+        start = torch.rand(wl.n, generator=gen, device=device) < 1.0 / wl.runs
+        run = torch.cumsum(start.to(torch.int64), 0)                          # run index of every token
+        nrun = int(run[-1].item()) + 1
+        # a random subset of topk groups per run and per token: the topk smallest of K uniform draws
+        pick = lambda rows: (torch.rand((rows, wl.K), generator=gen, device=device).argsort(dim=1) < wl.topk)
+        of_run, own = pick(nrun), pick(wl.n)
+        stray = torch.rand(wl.n, generator=gen, device=device) < wl.flip
+        member = torch.where(stray[:, None], own, of_run[run]).to(torch.float32)
     Q = torch.empty((wl.Hq, wl.n, wl.D), dtype=torch.bfloat16, device=device)
     K = torch.empty((wl.Hkv, wl.n, wl.D), dtype=torch.bfloat16, device=device)
     V = torch.empty((wl.Hkv, wl.n, wl.D), dtype=torch.bfloat16, device=device)
+    def mean_of(hk):
+        if z is not None:
+            return 2.0 * C[hk][z]
+        if member is not None:
+            return wl.signal * (member @ C[hk])
+        return None
     for h in range(wl.Hq):
-        mean = 2.0 * C[h // wl.G][z] if z is not None else None
-        Q[h] = _randn_bf16((wl.n, wl.D), gen, device, mean)
+        Q[h] = _randn_bf16((wl.n, wl.D), gen, device, mean_of(h // wl.G))
     for hk in range(wl.Hkv):
-        mean = 2.0 * C[hk][z] if z is not None else None
-        K[hk] = _randn_bf16((wl.n, wl.D), gen, device, mean)
+        K[hk] = _randn_bf16((wl.n, wl.D), gen, device, mean_of(hk))
     for hk in range(wl.Hkv):
         V[hk] = _randn_bf16((wl.n, wl.D), gen, device)
     return Q, K, V, C

@@ -63,3 +63,20 @@ def test_metric_point_128k():
 def test_cfg5_one_million_tokens():
     stats, frac = run_sampled("cfg5", 256)
     assert 0.82 < frac < 0.85
+
+
+@pytest.mark.parametrize("name,lo,hi", [("Mruns", 0.80, 0.90), ("Mruns1", 0.22, 0.32)])
+def test_run_structured_memberships_at_the_metric_shape(name, lo, hi):
+    """memberships coherent over positions: in the original layout whole far tiles die (skipped) and others are
+    attended without any mask; sampled rows against the oracle, tile counters against what the draw implies"""
+    stats, frac = run_sampled(name, 64)
+    assert lo < frac < hi
+    wl = fi.WORKLOADS[name]
+    Q, K, V, C = fi.make_inputs(wl, "cuda")
+    mq, _ = gpu_assign(wl, Q, C, wl.Hq)
+    mk, _ = gpu_assign(wl, K, C, wl.Hkv)
+    ws, L = gpu_tiles(wl, mq, mk, 0)
+    far, live, full = fb.ws_view(ws, L.counters, 8, torch.int64)[:3].tolist()
+    assert 0 < full < live < far
+    assert live < (0.95 if wl.topk == 2 else 0.6) * far          # a good part of the far tiles is never visited
+    assert full > 0.2 * live                                      # and a good part of the rest needs no mask
