@@ -181,7 +181,7 @@ def run_sweep(args):
             reps = 3 if n <= 262144 else 1
             row = dict(sweep=True, n=n, K=K, topk=topk, window=wl.window, Hq=32, Hkv=8, D=128)
             row["dense_ms"] = timed(lambda: fb.focus_attn_fwd(shape, Q, Kt, V, None, None, None, 0, O, lse, status), reps)
-            for layout, name in ((0, "original"), (1, "sorted"), (3, "sorted_local")):
+            for layout, name in ((0, "original"), (1, "sorted"), (3, "sorted_local"), (4, "group_major")):
                 ws = fb.alloc_workspace(shape, layout)
                 row[f"tiles_{name}_ms"] = timed(lambda: fb.focus_build_tiles(shape, mq, mk, layout, ws), reps)
                 row[f"{name}_ms"] = timed(lambda: fb.focus_attn_fwd(shape, Q, Kt, V, mq, mk, ws, layout, O, lse, status), reps)
@@ -193,7 +193,7 @@ def run_sweep(args):
                 del ws
             assert status[0].item() == 0, status.tolist()
             best = min(row["original_ms"] + row["tiles_original_ms"], row["sorted_ms"] + row["tiles_sorted_ms"],
-                       row["sorted_local_ms"] + row["tiles_sorted_local_ms"])
+                       row["sorted_local_ms"] + row["tiles_sorted_local_ms"], row["group_major_ms"] + row["tiles_group_major_ms"])
             row["auto_layout"] = fb.focus_tiles_layout_of(shape, fb.FOCUS_LAYOUT_AUTO).layout
             row["speedup_vs_dense"] = row["dense_ms"] / best
             row["kept_tflops_best"] = 4.0 * wl.D * row["kept_fraction"] * wl.dense_pairs() / (best * 1e-3) / 1e12
@@ -210,7 +210,8 @@ def main():
     ap.add_argument("--impl", default="focus", choices=["focus", "reference"])
     ap.add_argument("--workload", default="M128k")
     ap.add_argument("--layout", type=int, default=2, help="0 = original token order, 1 = class-sorted (group-permuted), 2 = chosen by the library from the shape, "
-                                                           "3 = class-sorted for sharing pairs + window pass in token order")
+                                                           "3 = class-sorted for sharing pairs + window pass in token order, "
+                                                           "4 = group-major key lists for sharing pairs + window pass")
     ap.add_argument("--ref-rows", type=int, default=2048, help="oracle rows per step (reference arm)")
     ap.add_argument("--cpu-rows", type=int, default=24576, help="oracle rows of the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -262,7 +263,7 @@ def main():
     status = torch.zeros(4, dtype=torch.int32, device="cuda")
     # assign x2, build_tiles (4 kernels; class-sorted: + 6 per side + ranges + order), attention (+ 3 gathers)
     # layout 3: + fill, second attention launch, merge
-    launches_per_step = 2 + 4 + 1 + (14 + 3 if layout in (1, 3) else 0) + (3 if layout == 3 else 0)
+    launches_per_step = 2 + 4 + 1 + (14 + 3 if layout in (1, 3, 4) else 0) + (3 if layout in (3, 4) else 0)
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
     marks = []
@@ -466,7 +467,7 @@ def main():
                         parallelism=("single GPU" if world == 1 else
                                      f"{world} replicas, no collective" if args.scaling == "weak" else
                                      f"KV heads split over {world} ranks, no collective"),
-                        softcap=wl.softcap, layout=["original", "class-sorted", None, "class-sorted + window pass"][layout],
+                        softcap=wl.softcap, layout=["original", "class-sorted", None, "class-sorted + window pass", "group-major keys + window pass"][layout],
                         l2="inputs larger than L2 (Q+K+V+O = %.2f GiB); no flush between steps" %
                            ((2 * Q.numel() + 2 * K.numel()) * 2 / 2**30)),
             clocks=clocks,

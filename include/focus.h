@@ -89,6 +89,15 @@ typedef struct {
  * and "Merge").  With many small classes the sorted order scatters the window of a query block over a wide range
  * of every other class; the separate pass reads the window once, in token order. */
 #define FOCUS_LAYOUT_SORTED_LOCAL 3
+/* Group-major keys: queries are sorted by class as above, but the keys of a KV head are laid out as K lists, list g
+ * holding (in token order) every key that is a member of group g -- a key with several groups is listed once per
+ * group.  A block of sorted queries walks the lists of its own groups only, and a pair that shares more than one
+ * group is attended under the lowest shared group (in the higher list the key is masked out for that row), so every
+ * sharing pair is computed exactly once; the pairs attended only because of the window come from the same second pass
+ * in token order as with FOCUS_LAYOUT_SORTED_LOCAL.  With top-k > 1 there are K lists of about n*topk/K keys instead
+ * of C(K, topk) class segments of about n/C(K, topk): the padding and the cut tiles at segment ends, which dominate
+ * when classes are many and small, fall away, at the price of listing (and staging) every key topk times. */
+#define FOCUS_LAYOUT_GROUP_MAJOR 4
 
 /*
  * Byte offsets of the arrays inside a tiles workspace (a pure function of shape and layout;
@@ -108,10 +117,13 @@ typedef struct {
     size_t live_cnt;   /* int32  [B*Hq][nqt]: popcount of the row of `live` */
     size_t kany, kall; /* uint32 [B*Hkv][K][nkw]: bit b set when key tile b holds a member of group g / only members of g */
     /* class-sorted layouts only (0 otherwise) */
-    int32_t nqp, nkp;  /* capacity of the sorted arrays in rows (multiples of 256): n + room for padding every class segment */
+    int32_t nqp, nkp;  /* capacity of the sorted arrays in rows (multiples of 256): n + room for padding every class segment;
+                          group-major keys: n*topk + room for padding every list */
     size_t ncls_q, ncls_k;   /* int32 [B*Hq], [B*Hkv]: distinct mask values of the head */
     size_t cls_q, cls_k;     /* uint32 [heads][FOCUS_MAX_CLASSES]: the mask values, ascending */
     size_t cnt_q, cnt_k;     /* int32 [heads][FOCUS_MAX_CLASSES]: tokens of each class */
+    /* (group-major keys: "class" j of the key side is group j -- ncls_k = K, cls_k[j] = 1 << j, cnt_k / seg_k / perm_k
+       describe the K lists) */
     size_t seg_q, seg_k;     /* int32 [heads][FOCUS_MAX_CLASSES+1]: first sorted slot of each class segment; query
                                 segments are padded to multiples of 256 slots, key segments to multiples of 128;
                                 entry [ncls] is the number of slots in use */
@@ -121,9 +133,12 @@ typedef struct {
                                 (128 slots) of each key class that a block of 256 sorted queries must visit */
     size_t order;            /* int32 [B*Hkv][(Hq/Hkv)*(nqp/256)][2]: (query head, query block) pairs of each KV head
                                 group, most key tiles first */
+    size_t gbits_s;          /* FOCUS_LAYOUT_GROUP_MAJOR only: uint32 [B*Hkv][nkp/128][K][4], bit j of word j/32 set when
+                                entry 128*b + j of the key lists is a member of group g (like gbits, in list order) */
     size_t qs, ks, vs;       /* bf16 sorted copies [B*Hq][nqp][D], [B*Hkv][nkp][D] x2, filled by focus_attn_fwd */
     size_t scratch;          /* build-time scratch (hash sets of mask values, chunk histograms, block costs) */
-    /* FOCUS_LAYOUT_SORTED_LOCAL only (0 otherwise): the two partial results, kept in fp32 until they are joined */
+    /* FOCUS_LAYOUT_SORTED_LOCAL and FOCUS_LAYOUT_GROUP_MAJOR only (0 otherwise): the two partial results, kept in fp32
+       until they are joined */
     size_t o_sorted;         /* fp32 [B*Hq][n][D]: class-sorted pass (its logsumexp goes to the caller's lse) */
     size_t o_local;          /* fp32 [B*Hq][n][D]: window pass */
     size_t lse_local;        /* fp32 [B*Hq][n] */

@@ -32,6 +32,11 @@ Passages of the paper each function follows:
                         combined with Appendix C's mask (same-class-sharing keys up to the block's last
                         position; other keys only inside the window).
 
+* ``group_major_layout`` the same Sec. 2 sort with a token that belongs to several groups (top-k > 1, Sec. 3.6)
+                        listed once per group: K key lists in token order; a block of sorted queries reads the lists
+                        of its own groups up to its last position, and a pair sharing several groups is attended under
+                        the lowest shared one.  Covers exactly the sharing pairs of Appendix C's mask, each once.
+
 * ``router_scores``     Sec. 2 "Learned grouping", the argument of Eq. 1's normalisation: (W_g h_i) . C_g.
 * ``sinkhorn``          Sec. 2 "Learned grouping", the two-step Sinkhorn normalisation: exponentiate the scores
                         over the temperature, then N times divide by the sums over tokens and by the sums over
@@ -355,6 +360,55 @@ def sorted_layout(mq_h: np.ndarray, mk_h: np.ndarray, window: int, pad_q: int = 
                 ranges[blk, jk] = ((seg_k[jk] + idx.min()) // tile, (seg_k[jk] + idx.max()) // tile + 1)
     return dict(cls_q=cls_q, cnt_q=cnt_q, seg_q=seg_q, perm_q=perm_q, cls_k=cls_k, cnt_k=cnt_k, seg_k=seg_k,
                 perm_k=perm_k, ranges=ranges)
+
+
+def group_major_layout(mq_h: np.ndarray, mk_h: np.ndarray, K: int, pad_q: int = 256, pad_k: int = 128, tile: int = 128):
+    """Group-major key lists of one (query head, KV head) pair, written from their definition.
+
+    Queries: stably sorted by mask value, class segments padded to ``pad_q`` (padding -1), as in ``sorted_layout``.
+    Keys: list g (g = 0..K-1) holds the positions of the keys that are members of group g, ascending, padded to a
+    multiple of ``pad_k`` with INT32_MAX; the lists follow one another.  ``gbits`` [tiles, K, tile] says for every
+    list entry which groups its key belongs to.  ``ranges`` [nblk, K, 2]: for a block of ``pad_q`` sorted queries of
+    class c and every group g in c, the tiles of list g (first, one past last) that hold a key at or before the
+    block's last position; (0, 0) otherwise.  ``attended(i_class, g, entry_mask)``: inside list g a row of class c
+    attends an entry iff g is the lowest group the two share.
+    """
+    mq_h = np.asarray(mq_h, np.uint32); mk_h = np.asarray(mk_h, np.uint32)
+    perm, cls_q, cnt_q = class_sort(mq_h)
+    seg_q = np.zeros(len(cls_q) + 1, np.int64)
+    seg_q[1:] = np.cumsum((cnt_q + pad_q - 1) // pad_q * pad_q)
+    perm_q = np.full(int(seg_q[-1]), -1, np.int64)
+    src = 0
+    for c in range(len(cls_q)):
+        perm_q[seg_q[c]:seg_q[c] + cnt_q[c]] = perm[src:src + cnt_q[c]]
+        src += cnt_q[c]
+    lists = [np.nonzero((mk_h >> g) & 1)[0].astype(np.int64) for g in range(K)]
+    cnt_k = np.array([len(l) for l in lists], np.int64)
+    seg_k = np.zeros(K + 1, np.int64)
+    seg_k[1:] = np.cumsum((cnt_k + pad_k - 1) // pad_k * pad_k)
+    perm_k = np.full(int(seg_k[-1]), np.iinfo(np.int32).max, np.int64)
+    for g in range(K):
+        perm_k[seg_k[g]:seg_k[g] + cnt_k[g]] = lists[g]
+    ntile = len(perm_k) // tile
+    gbits = np.zeros((ntile, K, tile), bool)
+    real = perm_k < len(mk_h)
+    member = np.zeros((len(perm_k), K), bool)
+    member[real] = ((mk_h[perm_k[real]][:, None] >> np.arange(K)[None, :]) & 1).astype(bool)
+    gbits[:] = member.reshape(ntile, tile, K).transpose(0, 2, 1)
+    nblk = int(seg_q[-1]) // pad_q
+    ranges = np.zeros((nblk, K, 2), np.int64)
+    for blk in range(nblk):
+        rows = perm_q[blk * pad_q:(blk + 1) * pad_q]
+        rows = rows[rows >= 0]
+        jq = int(np.searchsorted(seg_q, blk * pad_q, side="right")) - 1
+        pmax = int(rows.max())
+        for g in range(K):
+            if (int(cls_q[jq]) >> g) & 1:
+                hi = int(np.count_nonzero(lists[g] <= pmax))
+                if hi:
+                    ranges[blk, g] = (seg_k[g] // tile, (seg_k[g] + hi - 1) // tile + 1)
+    return dict(cls_q=cls_q, cnt_q=cnt_q, seg_q=seg_q, perm_q=perm_q, cnt_k=cnt_k, seg_k=seg_k, perm_k=perm_k,
+                gbits=gbits, ranges=ranges)
 
 
 def assign_hidden(h_bits: np.ndarray, Wg: np.ndarray, C: np.ndarray, topk: int, bias=None):

@@ -16,6 +16,7 @@ FOCUS_LAYOUT_ORIGINAL = 0
 FOCUS_LAYOUT_CLASS_SORTED = 1
 FOCUS_LAYOUT_AUTO = 2
 FOCUS_LAYOUT_SORTED_LOCAL = 3
+FOCUS_LAYOUT_GROUP_MAJOR = 4
 FOCUS_MAX_CLASSES = 64
 
 
@@ -39,7 +40,7 @@ class focus_tiles_layout(C.Structure):
                 ("ncls_q", C.c_size_t), ("ncls_k", C.c_size_t), ("cls_q", C.c_size_t), ("cls_k", C.c_size_t),
                 ("cnt_q", C.c_size_t), ("cnt_k", C.c_size_t),
                 ("seg_q", C.c_size_t), ("seg_k", C.c_size_t), ("perm_q", C.c_size_t), ("perm_k", C.c_size_t),
-                ("qrange", C.c_size_t), ("order", C.c_size_t), ("qs", C.c_size_t), ("ks", C.c_size_t),
+                ("qrange", C.c_size_t), ("order", C.c_size_t), ("gbits_s", C.c_size_t), ("qs", C.c_size_t), ("ks", C.c_size_t),
                 ("vs", C.c_size_t), ("scratch", C.c_size_t), ("o_sorted", C.c_size_t), ("o_local", C.c_size_t),
                 ("lse_local", C.c_size_t)]
 

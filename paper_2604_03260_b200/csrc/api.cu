@@ -106,9 +106,12 @@ static int layout_of(const focus_shape* s, int layout, focus_tiles_layout* L) {
     if (rc) return rc;
     if (!L) return fail(FOCUS_ERR_INVALID_ARG, "out is NULL");
     if (layout == FOCUS_LAYOUT_AUTO) layout = choose_layout(s);
-    if (layout != FOCUS_LAYOUT_ORIGINAL && layout != FOCUS_LAYOUT_CLASS_SORTED && layout != FOCUS_LAYOUT_SORTED_LOCAL)
+    if (layout != FOCUS_LAYOUT_ORIGINAL && !layout_is_sorted(layout))
         return fail(FOCUS_ERR_INVALID_ARG,
-                    "layout must be 0 (original), 1 (class-sorted), 2 (chosen by the library) or 3 (class-sorted + window pass)");
+                    "layout must be 0 (original), 1 (class-sorted), 2 (chosen by the library), 3 (class-sorted + window pass) "
+                    "or 4 (group-major keys + window pass)");
+    if (layout == FOCUS_LAYOUT_GROUP_MAJOR && group_major_capacity(s) > (1ll << 30))
+        return fail(FOCUS_ERR_UNSUPPORTED, "group-major layout: n * topk is too large");
     memset(L, 0, sizeof *L);
     const size_t HQ = (size_t)s->batch * s->Hq, HK = (size_t)s->batch * s->Hkv;
     L->layout = layout;
@@ -127,9 +130,9 @@ static int layout_of(const focus_shape* s, int layout, focus_tiles_layout* L) {
     L->live_cnt = take(HQ * L->nqt * 4);
     L->kany = take(HK * (size_t)s->K * L->nkw * 4);
     L->kall = take(HK * (size_t)s->K * L->nkw * 4);
-    if (layout == FOCUS_LAYOUT_CLASS_SORTED || layout == FOCUS_LAYOUT_SORTED_LOCAL) {
+    if (layout_is_sorted(layout)) {
         L->nqp = sorted_capacity(s->n);
-        L->nkp = sorted_capacity(s->n);
+        L->nkp = layout == FOCUS_LAYOUT_GROUP_MAJOR ? (int)group_major_capacity(s) : sorted_capacity(s->n);
         L->ncls_q = take(HQ * 4);
         L->ncls_k = take(HK * 4);
         L->cls_q = take(HQ * FOCUS_MAX_CLASSES * 4);
@@ -142,12 +145,13 @@ static int layout_of(const focus_shape* s, int layout, focus_tiles_layout* L) {
         L->perm_k = take(HK * (size_t)L->nkp * 4);
         L->qrange = take(HQ * (size_t)(L->nqp / 256) * FOCUS_MAX_CLASSES * 2 * 4);
         L->order = take(HQ * (size_t)(L->nqp / 256) * 2 * 4);
+        if (layout == FOCUS_LAYOUT_GROUP_MAJOR) L->gbits_s = take(HK * (size_t)(L->nkp / 128) * (size_t)s->K * 4 * 4);
         L->qs = take(HQ * (size_t)L->nqp * s->D * 2);
         L->ks = take(HK * (size_t)L->nkp * s->D * 2);
         L->vs = take(HK * (size_t)L->nkp * s->D * 2);
         L->scratch = take(sorted_scratch_bytes(s));
     }
-    if (layout == FOCUS_LAYOUT_SORTED_LOCAL) {
+    if (layout_has_window_pass(layout)) {
         L->o_sorted = take(HQ * (size_t)s->n * s->D * 4);
         L->o_local = take(HQ * (size_t)s->n * s->D * 4);
         L->lse_local = take(HQ * (size_t)s->n * 4);
@@ -266,7 +270,8 @@ int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, const uint32
     layout = L.layout;                     // FOCUS_LAYOUT_AUTO resolved
     if (layout == FOCUS_LAYOUT_CLASS_SORTED || layout == FOCUS_LAYOUT_SORTED_LOCAL) {
         // masks with exactly topk bits have C(K, topk) values; more than the class table holds is refused here,
-        // other mask patterns with too many values are caught on the device (counters[4], then dev_status)
+        // other mask patterns with too many values are caught on the device (counters[4], then dev_status).
+        // (Group-major keys need the table for the query side only: checked on the device.)
         double classes = 1.0;
         for (int j = 0; j < shape->topk; ++j) classes = classes * (shape->K - j) / (j + 1);
         if (classes > (double)FOCUS_MAX_CLASSES + 0.5)

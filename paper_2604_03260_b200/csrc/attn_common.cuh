@@ -86,6 +86,8 @@ struct AttnParams {
     // window pass of the split layout: only the tiles that reach into the window, only pairs WITHOUT a shared group
     // class-sorted pass of the split layout: only pairs WITH a shared group (the window pass covers the others)
     int share_only;
+    // group-major keys: bitmaps of the list entries per group, [B*Hkv][nkp/128][K][4] (nullptr in the other layouts)
+    const uint32_t* gbits_s;
     int local_only;
     float* o32;              // partial passes: O in fp32, rows [B*Hq][n][D], instead of bf16 to `o`
     unsigned long long wait_limit_ns;   // bound of every wait inside the kernel
@@ -286,5 +288,24 @@ __device__ __forceinline__ void build_tile_mask_sorted(TileMask& tm, int w, cons
         }
     }
 }
+
+// Group-major keys: the tile belongs to the list of group g.  A key that shares a LOWER group with the row is attended
+// under that lower group's list, so here it is masked out: `lower` = the row's groups below g, `gb` = the tile's
+// per-group bitmaps.  Every sharing pair is then computed exactly once.
+__device__ __forceinline__ void exclude_lower_groups(TileMask& tm, const uint32_t* __restrict__ gb, uint32_t lower, int K) {
+    uint32_t ex[4] = {0u, 0u, 0u, 0u};
+    for (uint32_t rem = lower; rem; rem &= rem - 1) {
+        const int a = __ffs(rem) - 1;
+        if (a < K) {
+            const uint4 t = __ldg(reinterpret_cast<const uint4*>(gb + a * 4));
+            ex[0] |= t.x; ex[1] |= t.y; ex[2] |= t.z; ex[3] |= t.w;
+        }
+    }
+    if (ex[0] | ex[1] | ex[2] | ex[3]) {
+        tm.masked = true;
+        tm.kw[0] &= ~ex[0]; tm.kw[1] &= ~ex[1]; tm.kw[2] &= ~ex[2]; tm.kw[3] &= ~ex[3];
+    }
+}
+
 
 }  // namespace focus

@@ -451,6 +451,8 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     const bool share = (mi & __ldg(p.cls_k + (size_t)hk * FOCUS_MAX_CLASSES + walk.jk)) != 0u;
                     build_tile_mask_sorted(tm, p.w, p.perm_k + (size_t)hk * p.nkp + (size_t)kb * 128, share,
                                            valid ? (int)i : -1, wmin, wmax, !p.share_only);
+                    if (p.gbits_s && !tm.all_masked)
+                        exclude_lower_groups(tm, p.gbits_s + ((size_t)hk * (p.nkp / 128) + kb) * p.K * 4, mi & ((1u << walk.jk) - 1u), p.K);
                 } else {
                     build_tile_mask(tm, p, a, kb, i, mi, aq, f_x, hk);
                 }
@@ -697,8 +699,7 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
     using C = AttnCfg<D, GATE>;
     CUtensorMap tq, tk, tv;
     int rc;
-    const bool sorted = a.ws && !a.local_pass &&
-                        (a.L.layout == FOCUS_LAYOUT_CLASS_SORTED || a.L.layout == FOCUS_LAYOUT_SORTED_LOCAL);
+    const bool sorted = a.ws && !a.local_pass && layout_is_sorted(a.L.layout);
     if (sorted) {
         // gather Q, K, V into the sorted order kept in the workspace; the kernel reads the copies
         char* ws = const_cast<char*>(a.ws);
@@ -745,7 +746,8 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
     p.counters = a.ws ? reinterpret_cast<const unsigned long long*>(a.ws + a.L.counters) : nullptr;
     p.gate_g = a.gate_g; p.gate_ld = a.gate_ld; p.gate_hl = 0.5f * a.gate_lambda;
     p.local_only = a.local_pass ? 1 : 0;
-    p.share_only = (sorted && a.L.layout == FOCUS_LAYOUT_SORTED_LOCAL) ? 1 : 0;
+    p.share_only = (sorted && layout_has_window_pass(a.L.layout)) ? 1 : 0;
+    p.gbits_s = (sorted && a.L.layout == FOCUS_LAYOUT_GROUP_MAJOR) ? reinterpret_cast<const uint32_t*>(a.ws + a.L.gbits_s) : nullptr;
     p.o32 = a.o32;
     p.wait_limit_ns = a.wait_limit_ns;
     p.stall_at = a.stall_at;
@@ -765,7 +767,7 @@ static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
 static int launch_attn_one(const AttnArgs& a, cudaStream_t st);
 
 int launch_attn_sm100(const AttnArgs& a, cudaStream_t st) {
-    if (a.ws && a.L.layout == FOCUS_LAYOUT_SORTED_LOCAL && !a.local_pass) {
+    if (a.ws && layout_has_window_pass(a.L.layout) && !a.local_pass) {
         // (1) sharing pairs in the class-sorted order -> o, lse; rows of blocks without key tiles keep lse = -inf
         // (2) window-only pairs in token order -> workspace; (3) join through the logsumexps
         char* ws = const_cast<char*>(a.ws);

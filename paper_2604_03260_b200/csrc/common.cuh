@@ -29,6 +29,14 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // layout-1 padded sorted length: room for every class segment to be rounded up to 256 slots
 inline int sorted_capacity(int n) { return (int)align_up((size_t)n + (size_t)FOCUS_MAX_CLASSES * 255, 256); }
+// group-major keys: every key once per group it belongs to (topk of them), every list padded to 128 slots
+inline long long group_major_capacity(const focus_shape* s) {
+    return (long long)align_up((size_t)s->n * (size_t)s->topk + (size_t)s->K * 127, 256);
+}
+inline bool layout_is_sorted(int layout) {
+    return layout == FOCUS_LAYOUT_CLASS_SORTED || layout == FOCUS_LAYOUT_SORTED_LOCAL || layout == FOCUS_LAYOUT_GROUP_MAJOR;
+}
+inline bool layout_has_window_pass(int layout) { return layout == FOCUS_LAYOUT_SORTED_LOCAL || layout == FOCUS_LAYOUT_GROUP_MAJOR; }
 
 // class-sorted layout, build-time scratch: per head a hash set of mask values (256 x 8 bytes), per head and
 // chunk of 1024 tokens a histogram over classes, and per query block its number of key tiles

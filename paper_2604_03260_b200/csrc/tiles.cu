@@ -185,7 +185,7 @@ int launch_build_tiles(const focus_shape* s, const uint32_t* mq, const uint32_t*
                                                  reinterpret_cast<int32_t*>(ws + L.live_cnt),
                                                  reinterpret_cast<unsigned long long*>(ws + L.counters));
     if ((rc = check_cuda(cudaGetLastError(), "build_tiles kernels"))) return rc;
-    if (layout == FOCUS_LAYOUT_CLASS_SORTED || layout == FOCUS_LAYOUT_SORTED_LOCAL)
+    if (layout_is_sorted(layout))
         return launch_build_tiles_sorted(s, mq, mk, L, ws, st);
     return FOCUS_OK;
 }

@@ -112,7 +112,7 @@ chunk_hist_kernel(const uint32_t* __restrict__ m, int n, const uint32_t* __restr
 // totals and padded segment starts
 __global__ void __launch_bounds__(MAXC)
 scan_chunks_kernel(int32_t* __restrict__ hist, int nchunk, const int32_t* __restrict__ ncls, int pad,
-                   int32_t* __restrict__ cnt, int32_t* __restrict__ seg) {
+                   int32_t* __restrict__ cnt, int32_t* __restrict__ seg, int npad, unsigned long long* counters) {
     __shared__ int tot[MAXC];
     const int head = blockIdx.x, c = threadIdx.x;
     int run = 0;
@@ -132,6 +132,8 @@ scan_chunks_kernel(int32_t* __restrict__ hist, int nchunk, const int32_t* __rest
             seg[(size_t)head * (MAXC + 1) + j] = s;
             if (j < nc) s += (tot[j] + pad - 1) / pad * pad;
         }
+        if (s > npad) atomicAdd(&counters[4], 1ull);      // more entries than the sorted arrays hold (group-major lists of
+                                                          // masks with more than topk bits): the attention kernel refuses
     }
 }
 
@@ -174,6 +176,83 @@ scatter_kernel(const uint32_t* __restrict__ m, int n, const uint32_t* __restrict
         const int slot = seg[(size_t)head * (MAXC + 1) + ci] + base[((size_t)head * nchunk + chunk) * MAXC + ci] +
                          wcnt[warp][ci] + rank;
         if (slot < npad) perm[(size_t)head * npad + slot] = t;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// 2b. group-major keys: K lists per KV head, list g = the keys that are members of group g, in token order.
+// "Class" j of the key side is group j, so that the range and attention code reads the lists like class segments.
+// ---------------------------------------------------------------------------------------------
+__global__ void group_classes_kernel(int heads, int K, uint32_t* __restrict__ cls, int32_t* __restrict__ ncls) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < heads * MAXC) cls[i] = (i % MAXC) < K ? 1u << (i % MAXC) : 0u;
+    if (i < heads) ncls[i] = K;
+}
+
+__global__ void __launch_bounds__(SORT_CHUNK)
+group_hist_kernel(const uint32_t* __restrict__ m, int n, int K, int nchunk, int32_t* __restrict__ hist) {
+    __shared__ int h[MAXC];
+    const int head = blockIdx.y, chunk = blockIdx.x;
+    if (threadIdx.x < MAXC) h[threadIdx.x] = 0;
+    __syncthreads();
+    const int t = chunk * SORT_CHUNK + threadIdx.x;
+    const uint32_t v = t < n ? m[(size_t)head * n + t] : 0u;
+    for (int g = 0; g < K; ++g) {
+        const unsigned int b = __ballot_sync(0xffffffffu, (v >> g) & 1u);
+        if ((threadIdx.x & 31) == 0 && b) atomicAdd(&h[g], __popc(b));
+    }
+    __syncthreads();
+    if (threadIdx.x < MAXC) hist[((size_t)head * nchunk + chunk) * MAXC + threadIdx.x] = h[threadIdx.x];
+}
+
+// stable scatter into the lists: a key goes to the list of every group it belongs to
+__global__ void __launch_bounds__(SORT_CHUNK)
+group_scatter_kernel(const uint32_t* __restrict__ m, int n, int K, int nchunk, const int32_t* __restrict__ base,
+                     const int32_t* __restrict__ seg, int npad, int32_t* __restrict__ perm) {
+    __shared__ int wcnt[SORT_CHUNK / 32][32];
+    const int head = blockIdx.y, chunk = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t = chunk * SORT_CHUNK + threadIdx.x;
+    const uint32_t v = t < n ? m[(size_t)head * n + t] : 0u;
+    int rank[32];
+#pragma unroll
+    for (int g = 0; g < 32; ++g) {
+        const unsigned int b = g < K ? __ballot_sync(0xffffffffu, (v >> g) & 1u) : 0u;
+        rank[g] = __popc(b & ((1u << lane) - 1u));
+        if (lane == 0) wcnt[warp][g] = __popc(b);
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {                 // exclusive scan over the warps, per group
+        int run = 0;
+        for (int w = 0; w < SORT_CHUNK / 32; ++w) {
+            const int c = wcnt[w][threadIdx.x];
+            wcnt[w][threadIdx.x] = run;
+            run += c;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int g = 0; g < 32; ++g) {
+        if (g < K && ((v >> g) & 1u)) {
+            const int slot = seg[(size_t)head * (MAXC + 1) + g] + base[((size_t)head * nchunk + chunk) * MAXC + g] +
+                             wcnt[warp][g] + rank[g];
+            if (slot < npad) perm[(size_t)head * npad + slot] = t;
+        }
+    }
+}
+
+// block of 128 threads per (tile of the lists, KV head): per group the bitmap of entries that are members of it
+__global__ void __launch_bounds__(128)
+gbits_sorted_kernel(const uint32_t* __restrict__ m, int n, int K, const int32_t* __restrict__ perm, int npad,
+                    uint32_t* __restrict__ gbits_s) {
+    const int tile = blockIdx.x, head = blockIdx.y;
+    const int pos = perm[(size_t)head * npad + (size_t)tile * 128 + threadIdx.x];
+    const uint32_t v = (pos >= 0 && pos < n) ? m[(size_t)head * n + pos] : 0u;
+    uint32_t* gb = gbits_s + ((size_t)head * (npad / 128) + tile) * K * 4;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int g = 0; g < K; ++g) {
+        const uint32_t word = __ballot_sync(0xffffffffu, (v >> g) & 1u);
+        if (lane == 0) gb[g * 4 + warp] = word;
     }
 }
 
@@ -360,10 +439,20 @@ int launch_build_tiles_sorted(const focus_shape* s, const uint32_t* mq, const ui
         auto* seg = reinterpret_cast<int32_t*>(ws + (side ? L.seg_k : L.seg_q));
         auto* perm = reinterpret_cast<int32_t*>(ws + (side ? L.perm_k : L.perm_q));
         const int npad = side ? L.nkp : L.nqp;
+        if (side && L.layout == FOCUS_LAYOUT_GROUP_MAJOR) {
+            group_classes_kernel<<<cdiv(heads * MAXC, 256), 256, 0, st>>>(heads, s->K, cls, ncls);
+            group_hist_kernel<<<dim3(nchunk, heads), SORT_CHUNK, 0, st>>>(m, s->n, s->K, nchunk, hs);
+            scan_chunks_kernel<<<heads, MAXC, 0, st>>>(hs, nchunk, ncls, 128, cnt, seg, npad, counters);
+            fill_kernel<<<1184, 256, 0, st>>>(perm, (size_t)heads * npad, INT_MAX);
+            group_scatter_kernel<<<dim3(nchunk, heads), SORT_CHUNK, 0, st>>>(m, s->n, s->K, nchunk, hs, seg, npad, perm);
+            gbits_sorted_kernel<<<dim3(npad / 128, heads), 128, 0, st>>>(m, s->n, s->K, perm, npad,
+                                                                         reinterpret_cast<uint32_t*>(ws + L.gbits_s));
+            continue;
+        }
         collect_classes_kernel<<<dim3(nchunk, heads), 256, 0, st>>>(m, s->n, tab);
         finalize_classes_kernel<<<heads, SORT_HASH, 0, st>>>(tab, cls, ncls, counters);
         chunk_hist_kernel<<<dim3(nchunk, heads), SORT_CHUNK, 0, st>>>(m, s->n, cls, ncls, nchunk, hs);
-        scan_chunks_kernel<<<heads, MAXC, 0, st>>>(hs, nchunk, ncls, side ? 128 : 256, cnt, seg);
+        scan_chunks_kernel<<<heads, MAXC, 0, st>>>(hs, nchunk, ncls, side ? 128 : 256, cnt, seg, npad, counters);
         fill_kernel<<<1184, 256, 0, st>>>(perm, (size_t)heads * npad, side ? INT_MAX : -1);
         scatter_kernel<<<dim3(nchunk, heads), SORT_CHUNK, 0, st>>>(m, s->n, cls, ncls, nchunk, hs, seg, npad, perm);
     }
@@ -375,7 +464,7 @@ int launch_build_tiles_sorted(const focus_shape* s, const uint32_t* mq, const ui
         reinterpret_cast<const int32_t*>(ws + L.cnt_k), reinterpret_cast<const int32_t*>(ws + L.seg_q),
         reinterpret_cast<const int32_t*>(ws + L.seg_k), reinterpret_cast<const int32_t*>(ws + L.perm_q),
         reinterpret_cast<const int32_t*>(ws + L.perm_k), reinterpret_cast<int32_t*>(ws + L.qrange), cost, counters,
-        L.layout == FOCUS_LAYOUT_SORTED_LOCAL ? 1 : 0);
+        layout_has_window_pass(L.layout) ? 1 : 0);
     order_kernel<<<HK, 1024, 0, st>>>(s->Hq, s->Hkv, s->Hq / s->Hkv, nqblk, L.nkp / 128, cost,
                                       reinterpret_cast<int32_t*>(ws + L.order));
     return check_cuda(cudaGetLastError(), "build_tiles (class-sorted) kernels");

@@ -110,11 +110,16 @@ def test_auto_layout_is_resolved_from_the_shape():
     s = fb.make_shape(32, 8, 131072, 128, 4, 2, 2048)
     assert fb.focus_tiles_workspace_bytes(s, fb.FOCUS_LAYOUT_AUTO) == fb.focus_tiles_workspace_bytes(s, 1)
     L = fb.focus_tiles_layout()
-    assert fb.lib().focus_tiles_layout_of(ctypes.byref(s), 4, ctypes.byref(L)) == -1
+    assert fb.lib().focus_tiles_layout_of(ctypes.byref(s), 5, ctypes.byref(L)) == -1
     # the split layout: the sorted arrays plus two fp32 partial results and one logsumexp per row
     L1, L3 = fb.focus_tiles_layout_of(s, 1), fb.focus_tiles_layout_of(s, 3)
     assert L3.layout == 3 and L3.qrange == L1.qrange and L1.o_sorted == 0 and L3.o_sorted >= L1.total_bytes
     assert L3.o_local - L3.o_sorted >= 32 * 131072 * 128 * 4 and L3.total_bytes - L3.lse_local >= 32 * 131072 * 4
+    # group-major keys: every key listed once per group (topk times), one bitmap set per list tile, same query side
+    L4 = fb.focus_tiles_layout_of(s, fb.FOCUS_LAYOUT_GROUP_MAJOR)
+    assert L4.layout == 4 and L4.nqp == L1.nqp and L4.nkp >= 2 * 131072 + 4 * 127 and L4.nkp % 256 == 0
+    assert L4.gbits_s > 0 and L4.qs - L4.gbits_s >= 8 * (L4.nkp // 128) * 4 * 16 and L1.gbits_s == 0 and L4.o_local > L4.o_sorted > 0
+    assert L4.vs - L4.ks >= 8 * L4.nkp * 128 * 2
 
 
 def test_training_forward_host_checks():

@@ -362,6 +362,53 @@ def test_class_sort_is_stable_and_preserves_kept_sets():
     assert np.array_equal(Ms, M[np.ix_(pq, pk)])
 
 
+@pytest.mark.parametrize("n,K,t", [(700, 4, 2), (900, 8, 2), (600, 6, 3), (500, 4, 1), (300, 5, 5)])
+def test_group_major_lists_cover_every_sharing_pair_exactly_once(n, K, t):
+    """walking, for every query, the lists of its own groups up to its position and attending an entry only under the
+    lowest shared group visits each causal pair with intersecting masks exactly once and no other pair; the listed
+    tile ranges contain all of them and end on a tile that holds one"""
+    rng = np.random.default_rng(n + K + t)
+    mq = np.array([sum(1 << int(g) for g in rng.choice(K, t, replace=False)) for _ in range(n)], np.uint32)
+    mk = np.array([sum(1 << int(g) for g in rng.choice(K, t, replace=False)) for _ in range(n)], np.uint32)
+    L = fo.group_major_layout(mq, mk, K)
+    share = ((mq[:, None] & mk[None, :]) != 0) & (np.arange(n)[None, :] <= np.arange(n)[:, None])     # explicit matrix
+    times = np.zeros((n, n), np.int64)
+    in_range = np.zeros((n, n), bool)
+    for blk in range(L["ranges"].shape[0]):
+        rows = L["perm_q"][blk * 256:(blk + 1) * 256]
+        rows = rows[rows >= 0]
+        jq = int(np.searchsorted(L["seg_q"], blk * 256, side="right")) - 1
+        assert (mq[rows] == L["cls_q"][jq]).all()
+        for g in range(K):
+            first, last = L["ranges"][blk, g]
+            if not (int(L["cls_q"][jq]) >> g) & 1:
+                assert first == last == 0
+                continue
+            if last > first:
+                assert first * 128 == L["seg_k"][g] and last * 128 <= L["seg_k"][g + 1]
+            slots = np.arange(first * 128, last * 128)
+            pos = L["perm_k"][slots]
+            real = pos < n
+            lower = int(L["cls_q"][jq]) & ((1 << g) - 1)
+            ent_mask = np.zeros(len(slots), np.int64)
+            ent_mask[real] = mk[pos[real]]
+            assert ((ent_mask[real] >> g) & 1).all()                       # the list holds members of g only
+            assert (np.diff(pos[real]) > 0).all()                          # in token order
+            ok_col = real & ((ent_mask & lower) == 0)                      # not attended under a lower shared group
+            for i in rows:
+                cols = pos[ok_col & (pos <= i)]
+                np.add.at(times[i], cols, 1)
+                in_range[i, pos[real & (pos <= i)]] = True
+            if last > first:                                               # the last listed tile holds a causal key of the block
+                assert (pos[(last - first - 1) * 128:][real[(last - first - 1) * 128:]] <= rows.max()).any()
+    assert np.array_equal(times, share.astype(np.int64))
+    # gbits is the membership of every list entry
+    flat = L["gbits"].transpose(0, 2, 1).reshape(-1, K)
+    real = L["perm_k"] < n
+    want = ((mk[L["perm_k"][real]][:, None] >> np.arange(K)[None, :]) & 1).astype(bool)
+    assert np.array_equal(flat[real], want) and not flat[~real].any()
+
+
 @pytest.mark.parametrize("n,K,t,w", [(700, 4, 2, 40), (1500, 4, 1, 100), (900, 8, 2, 0), (600, 2, 1, 1000)])
 def test_sorted_layout_ranges_cover_exactly_the_tiles_with_kept_pairs(n, K, t, w):
     """every kept pair of the explicit mask lies in a listed tile of its key class; the first and last listed
