@@ -46,6 +46,12 @@ Passages of the paper each function follows:
                         window keeps its score.  The equation is followed as printed, so the gate of two
                         orthogonal assignments is sigmoid(0) = 1/2 (the prose around it speaks of zero).
 
+* ``sinkhorn_backward`` / ``gated_attn_backward``
+                        the derivatives of the two functions above (chain rule through every division of the
+                        Sinkhorn steps; through the row softmax, the gate sigmoid(lambda g_i . g_j) and the score of
+                        Eq. 2).  No kernel computes them yet: they are the reference a backward pass would be
+                        checked against, pinned by finite differences and by automatic differentiation.
+
 Parity status: every function above is pinned by the CPU tests.  "parity unpinned": the paper's
 perplexity and benchmark numbers (datasets and trained weights are not available).
 """
@@ -483,3 +489,64 @@ def gated_attn(q_bits, k_bits, v_bits, g, lam, window, scale=None, rows=None):
             O[h, r] = (e / Z) @ V[h // G][causal]
             lse[h, r] = m + np.log(Z)
     return O, lse
+
+
+def sinkhorn_backward(S: np.ndarray, tau: float, iters: int, dG: np.ndarray) -> np.ndarray:
+    """d loss / d S for g = sinkhorn(S, tau, iters), given dG = d loss / d g  ([n, K] both).
+
+    Forward steps kept on a tape: Q0 = exp(S / tau); per iteration Y = X / colsum(X), then Z = Y / rowsum(Y).  For a
+    division by the sum over an axis, Z = X / sum(X):  dX = (dZ - sum(dZ * Z)) / sum(X) along that axis.
+    """
+    tau = float(tau)
+    X = np.exp(np.asarray(S, np.float64) / tau)
+    Q0 = X
+    tape = []
+    for _ in range(int(iters)):
+        c = X.sum(axis=0, keepdims=True); Y = X / c
+        r = Y.sum(axis=1, keepdims=True); Z = Y / r
+        tape.append((c, Y, r, Z))
+        X = Z
+    d = np.asarray(dG, np.float64).copy()
+    for c, Y, r, Z in reversed(tape):
+        d = (d - (d * Z).sum(axis=1, keepdims=True)) / r          # through the division by the row sums
+        d = (d - (d * Y).sum(axis=0, keepdims=True)) / c          # through the division by the column sums
+    return d * Q0 / tau
+
+
+def gated_attn_backward(q_bits, k_bits, v_bits, g, lam, window, dO, scale=None):
+    """Derivatives of ``gated_attn`` (all rows) with respect to Q, K, V and the soft assignments g.
+
+    dO float [Hq, n, D] = d loss / d O.  With p the row softmax of s_ij = scale * <q_i, k_j> * f_ij over j <= i,
+    f_ij = 1 inside the window and sigmoid(lam * <g_i, g_j>) beyond it:
+        dV_j += p_ij dO_i;   ds_ij = p_ij (<dO_i, v_j> - <dO_i, o_i>);
+        dq_i += ds_ij scale f_ij k_j;   dk_j += ds_ij scale f_ij q_i;
+        beyond the window: du_ij = ds_ij scale <q_i, k_j> f_ij (1 - f_ij) lam;   dg_i += du_ij g_j;   dg_j += du_ij g_i.
+    Query heads that share a KV head add into the same dK / dV rows; every head adds into dg.
+    Returns (dQ [Hq, n, D], dK [Hkv, n, D], dV [Hkv, n, D], dg [n, K]) in fp64.
+    """
+    Q = bf16_bits_to_f64(np.asarray(q_bits)); Kx = bf16_bits_to_f64(np.asarray(k_bits)); V = bf16_bits_to_f64(np.asarray(v_bits))
+    Hq, n, D = Q.shape
+    G = Hq // Kx.shape[0]
+    sc = 1.0 / np.sqrt(D) if scale is None else float(scale)
+    g = np.asarray(g, np.float64); dO = np.asarray(dO, np.float64); lam = float(lam)
+    dQ = np.zeros_like(Q); dK = np.zeros_like(Kx); dV = np.zeros_like(V); dg = np.zeros_like(g)
+    for i in range(n):
+        j = np.arange(i + 1)
+        aff = g[:i + 1] @ g[i]
+        far = (i - j) > window
+        f = np.where(far, 1.0 / (1.0 + np.exp(-lam * aff)), 1.0)
+        for h in range(Hq):
+            hk = h // G
+            qk = Kx[hk, :i + 1] @ Q[h, i]
+            s = sc * qk * f
+            e = np.exp(s - s.max())
+            p = e / e.sum()
+            o = p @ V[hk, :i + 1]
+            dV[hk, :i + 1] += p[:, None] * dO[h, i][None, :]
+            ds = p * (V[hk, :i + 1] @ dO[h, i] - dO[h, i] @ o)
+            dQ[h, i] += (ds * sc * f) @ Kx[hk, :i + 1]
+            dK[hk, :i + 1] += (ds * sc * f)[:, None] * Q[h, i][None, :]
+            du = np.where(far, ds * sc * qk * f * (1.0 - f) * lam, 0.0)
+            dg[i] += du @ g[:i + 1]
+            dg[:i + 1] += du[:, None] * g[i][None, :]
+    return dQ, dK, dV, dg

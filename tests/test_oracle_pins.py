@@ -597,3 +597,88 @@ def test_gated_attn_half_gate_is_half_scale():
     qb, kb, vb = bits(q), bits(k), rand_bits(rng, (H, n, 2))
     O, _ = fo.gated_attn(qb, kb, vb, np.zeros((n, 4)), 5.0, 0, scale=0.25)
     np.testing.assert_allclose(O, sdpa_causal(qb, kb, vb, 0.125), atol=1e-12)
+
+
+# ---------------------------------------------------------------- derivatives of the training-time forward (Sec. 2)
+def test_sinkhorn_backward_matches_finite_differences_and_autograd():
+    """the chain rule through the N column / row divisions against central differences of the oracle's own forward and
+    against automatic differentiation of the same steps written with torch"""
+    import torch
+    rng = np.random.default_rng(4)
+    n, K, tau, N = 9, 4, 0.7, 3
+    S = rng.standard_normal((n, K)) * 0.5
+    dG = rng.standard_normal((n, K))
+    got = fo.sinkhorn_backward(S, tau, N, dG)
+    num = np.zeros_like(S)
+    eps = 1e-6
+    for a in range(n):
+        for b in range(K):
+            Sp = S.copy(); Sp[a, b] += eps
+            Sm = S.copy(); Sm[a, b] -= eps
+            num[a, b] = ((fo.sinkhorn(Sp, tau, N) - fo.sinkhorn(Sm, tau, N)) * dG).sum() / (2 * eps)
+    assert np.abs(got - num).max() < 1e-7
+    St = torch.tensor(S, dtype=torch.float64, requires_grad=True)
+    Qt = torch.exp(St / tau)
+    for _ in range(N):
+        Qt = Qt / Qt.sum(dim=0, keepdim=True)
+        Qt = Qt / Qt.sum(dim=1, keepdim=True)
+    assert np.abs(Qt.detach().numpy() - fo.sinkhorn(S, tau, N)).max() < 1e-14
+    (Qt * torch.tensor(dG)).sum().backward()
+    assert np.abs(got - St.grad.numpy()).max() < 1e-12
+    # the assignments do not change when one group's scores are shifted by a constant (the first column division removes
+    # it): the gradient summed over the tokens of a column vanishes
+    assert np.abs(got.sum(axis=0)).max() < 1e-12
+
+
+@pytest.mark.parametrize("Hq,Hkv,w", [(2, 1, 1), (2, 2, 0), (4, 2, 3)])
+def test_gated_attention_backward_matches_autograd_and_finite_differences(Hq, Hkv, w):
+    """dQ, dK, dV and d(assignments) of Eq. 2's forward: automatic differentiation of the explicit dense formula
+    (whose forward equals the oracle's), plus central differences of the oracle's forward on a few entries"""
+    import torch
+    rng = np.random.default_rng(10 * Hq + w)
+    n, D, K, lam = 7, 4, 3, 3.0
+    bf = lambda x: torch.tensor(x).to(torch.bfloat16)
+    Qb, Kb, Vb = bf(rng.standard_normal((Hq, n, D))), bf(rng.standard_normal((Hkv, n, D))), bf(rng.standard_normal((Hkv, n, D)))
+    bits = lambda t: t.view(torch.int16).numpy().view(np.uint16)
+    g = rng.random((n, K)); g /= g.sum(axis=1, keepdims=True)
+    dO = rng.standard_normal((Hq, n, D))
+    dQ, dK, dV, dg = fo.gated_attn_backward(bits(Qb), bits(Kb), bits(Vb), g, lam, w, dO)
+    # explicit dense formula in torch
+    Qt = Qb.double().requires_grad_(True); Kt = Kb.double().requires_grad_(True); Vt = Vb.double().requires_grad_(True)
+    gt = torch.tensor(g, requires_grad=True)
+    G = Hq // Hkv
+    idx = torch.arange(n)
+    causal = idx[None, :] <= idx[:, None]
+    far = (idx[:, None] - idx[None, :]) > w
+    f = torch.where(far, torch.sigmoid(lam * (gt @ gt.T)), torch.ones((), dtype=torch.float64))
+    outs = []
+    for h in range(Hq):
+        s = (Qt[h] @ Kt[h // G].T) / D ** 0.5 * f
+        s = s.masked_fill(~causal, float("-inf"))
+        outs.append(torch.softmax(s, dim=1) @ Vt[h // G])
+    O = torch.stack(outs)
+    ref_O, _ = fo.gated_attn(bits(Qb), bits(Kb), bits(Vb), g, lam, w)
+    assert np.abs(O.detach().numpy() - ref_O).max() < 1e-12           # the same forward
+    (O * torch.tensor(dO)).sum().backward()
+    for got, want in ((dQ, Qt.grad), (dK, Kt.grad), (dV, Vt.grad), (dg, gt.grad)):
+        assert np.abs(got - want.numpy()).max() < 1e-11
+    # central differences of the oracle's forward with respect to a few assignment entries
+    eps = 1e-6
+    for a, b in ((0, 0), (n - 1, 1), (n // 2, 2)):
+        gp = g.copy(); gp[a, b] += eps
+        gm = g.copy(); gm[a, b] -= eps
+        num = ((fo.gated_attn(bits(Qb), bits(Kb), bits(Vb), gp, lam, w)[0] - fo.gated_attn(bits(Qb), bits(Kb), bits(Vb), gm, lam, w)[0]) * dO).sum() / (2 * eps)
+        assert abs(num - dg[a, b]) < 1e-6
+    if w >= n:
+        assert np.abs(dg).max() == 0.0
+
+
+def test_gated_attention_backward_without_distant_pairs_has_no_assignment_gradient():
+    rng = np.random.default_rng(2)
+    import torch
+    n, D = 5, 4
+    bits = lambda x: torch.tensor(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    q, k, v = bits(rng.standard_normal((1, n, D))), bits(rng.standard_normal((1, n, D))), bits(rng.standard_normal((1, n, D)))
+    g = rng.random((n, 2))
+    dQ, dK, dV, dg = fo.gated_attn_backward(q, k, v, g, 5.0, n, rng.standard_normal((1, n, D)))
+    assert np.abs(dg).max() == 0.0 and np.abs(dQ).max() > 0 and np.abs(dK).max() > 0 and np.abs(dV).max() > 0
