@@ -85,7 +85,7 @@ typedef struct {
 #define FOCUS_LAYOUT_AUTO 2
 /* Class-sorted layout for the pairs that share a group, plus a second pass in the original token order for the
  * pairs that are attended only because they lie inside the window (no shared group); the two partial results
- * cover disjoint sets of pairs and are joined through their logsumexps (paper Appendix C, "Disjoint decomposition"
+ * cover disjoint sets of pairs and are joined through their logsumexps (paper Appendix D, "Disjoint decomposition"
  * and "Merge").  With many small classes the sorted order scatters the window of a query block over a wide range
  * of every other class; the separate pass reads the window once, in token order. */
 #define FOCUS_LAYOUT_SORTED_LOCAL 3
@@ -215,7 +215,7 @@ FOCUS_API int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, co
 
 /*
  * focus_attn_fwd -- causal attention forward over the attended pairs (paper Sec. 2 and
- * Appendix C, first equation): pair (i, j) is attended iff
+ * Appendix D, first equation): pair (i, j) is attended iff
  *        j <= i  and  ( i - j <= window  or  mq[h,i] & mk[kv(h),j] != 0 ).
  * s_ij = scale*q_i.k_j (then softcap*tanh(s_ij/softcap) if softcap > 0);
  * lse_i = log sum_j exp(s_ij); o_i = sum_j exp(s_ij - lse_i) v_j over attended j: exact softmax,
@@ -237,8 +237,9 @@ FOCUS_API int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, co
  *               waiting for S, its partner thread or O), [2] = work item, [3] = CTA.  [0] = 2: a class-sorted layout was asked for
  *               but a head holds more than FOCUS_MAX_CLASSES distinct mask values (possible only with
  *               masks that do not come from a top-k rule); nothing was computed and O / lse were not
- *               written.  Pass a non-NULL dev_status with layouts 1 and 3 when the masks are not the
- *               library's own.  The caller zeroes it and reads it after synchronising.
+ *               written.  dev_status must not be NULL with a tiles workspace in any layout but
+ *               FOCUS_LAYOUT_ORIGINAL (FOCUS_ERR_INVALID_ARG otherwise).  The caller zeroes it and reads
+ *               it after synchronising.
  */
 FOCUS_API int focus_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k, focus_tensor v,
                    const uint32_t* mq, const uint32_t* mk, const void* tiles_ws, int32_t layout,
@@ -247,7 +248,7 @@ FOCUS_API int focus_attn_fwd(const focus_shape* shape, focus_tensor q, focus_ten
 /*
  * focus_decode_step -- one generation step: the newest token (position n-1, its key and value already appended
  * to the caches) as the only query, under the same rule as focus_attn_fwd (paper Sec. 2 "Efficiency at inference",
- * Appendix C first equation): key j is attended iff n-1-j <= window or mq_new[h] & mk[kv(h), j] != 0; exact softmax
+ * Appendix D first equation): key j is attended iff n-1-j <= window or mq_new[h] & mk[kv(h), j] != 0; exact softmax
  * over the attended keys; bf16 operands, fp32 accumulation, probabilities rounded to bf16 before P V.  The paper evaluates generation with the method but
  * gives no procedure; this is the forward rule applied to one row.  Only attended K/V rows are read from HBM.
  *   shape       n = cached tokens including the new one; Hq / Hkv <= 8

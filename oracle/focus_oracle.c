@@ -17,12 +17,12 @@
  *                              cosine between the head vector and the centroid (for unit
  *                              centroids it ranks groups exactly as Eq. 1's dot product does).
  *   focus_oracle_attn_rows  -- Sec. 2 (softmax(QK^T/sqrt(d))V restricted to attended pairs, exact
- *                              softmax with no renormalisation) with the hard mask of Appendix C
+ *                              softmax with no renormalisation) with the hard mask of Appendix D
  *                              (first equation): pair (i,j) is attended iff j <= i and (i-j <= w
  *                              or the two tokens share a group); "share a group" is the top-k
  *                              rule of Sec. 3.6 (membership sets intersect).
  * Parity status: both functions are pinned by the CPU tests (brute force with an explicit dense
- * mask, closed forms, reductions to textbook causal attention, the Appendix C two-set merge, a
+ * mask, closed forms, reductions to textbook causal attention, the Appendix D two-set merge, a
  * hand-worked case).  The paper's perplexity/benchmark numbers are "parity unpinned": they need
  * datasets and trained weights that are not available.
  */

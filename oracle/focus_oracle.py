@@ -14,14 +14,14 @@ Passages of the paper each function follows:
                         (row-softmax and the temperature do not change a row's ranking).  The optional per-group
                         bias is what Sinkhorn's column scaling leaves behind at inference: the balanced
                         assignment is diag(r) exp(S/tau) diag(c), whose row ranking is that of S + tau log c.
-* ``attn_rows``         Sec. 2 (exact softmax over attended pairs) + Appendix C, first equation
+* ``attn_rows``         Sec. 2 (exact softmax over attended pairs) + Appendix D, first equation
                         (the hard Focus mask), with "same group" read as "membership sets intersect".
-* ``dense_brute``       the O(n^2) masked reference the paper verifies against (Appendix C,
+* ``dense_brute``       the O(n^2) masked reference the paper verifies against (Appendix D,
                         "Empirical verification"): explicit n x n boolean matrix, textbook softmax.
-* ``ab_merge``          Appendix C "Disjoint decomposition" and "Merge": sets A (same-group causal)
+* ``ab_merge``          Appendix D "Disjoint decomposition" and "Merge": sets A (same-group causal)
                         and B (cross-group local) computed separately and joined through their
                         logsumexps.  Defined by the paper for single-group assignment only.
-* ``kept_pairs``        size of the attended set of Appendix C's mask (exact integer count).
+* ``kept_pairs``        size of the attended set of Appendix D's mask (exact integer count).
 * ``tile_reference``    the per-tile mask summaries and the far-tile liveness rule (a far tile can be
                         dropped when no query of the tile shares a group with any key of the tile);
                         this is the tile-level consequence of Sec. 2 "different-group distant pairs
@@ -29,13 +29,13 @@ Passages of the paper each function follows:
 * ``class_sort``        Sec. 2 "Sort tokens by group (stable sort preserves causal order)".
 * ``sorted_layout``     the padded class-sorted arrays and, per block of sorted queries and key class, the
                         range of sorted key tiles that can hold an attended pair -- the same Sec. 2 sort
-                        combined with Appendix C's mask (same-class-sharing keys up to the block's last
+                        combined with Appendix D's mask (same-class-sharing keys up to the block's last
                         position; other keys only inside the window).
 
 * ``group_major_layout`` the same Sec. 2 sort with a token that belongs to several groups (top-k > 1, Sec. 3.6)
                         listed once per group: K key lists in token order; a block of sorted queries reads the lists
                         of its own groups up to its last position, and a pair sharing several groups is attended under
-                        the lowest shared one.  Covers exactly the sharing pairs of Appendix C's mask, each once.
+                        the lowest shared one.  Covers exactly the sharing pairs of Appendix D's mask, each once.
 
 * ``router_scores``     Sec. 2 "Learned grouping", the argument of Eq. 1's normalisation: (W_g h_i) . C_g.
 * ``sinkhorn``          Sec. 2 "Learned grouping", the two-step Sinkhorn normalisation: exponentiate the scores
@@ -167,7 +167,7 @@ def attn_rows(q_bits, k_bits, v_bits, mq, mk, window, scale=None, softcap=0.0, r
 # ----------------------------------------------------------------------------------------------
 
 def kept_matrix(mq_h: np.ndarray, mk_h: np.ndarray, window: int) -> np.ndarray:
-    """Explicit n x n boolean mask of Appendix C's first equation for one (q head, kv head) pair."""
+    """Explicit n x n boolean mask of Appendix D's first equation for one (q head, kv head) pair."""
     n = mq_h.shape[0]
     i = np.arange(n)[:, None]
     j = np.arange(n)[None, :]
@@ -204,10 +204,10 @@ def dense_brute(q_bits, k_bits, v_bits, mq, mk, window, scale=None, softcap=0.0)
 
 
 def ab_merge(q_bits, k_bits, v_bits, g, window, scale=None, double_count=False):
-    """Appendix C two-set path for single-group assignment g [n] (one head, MHA).
+    """Appendix D two-set path for single-group assignment g [n] (one head, MHA).
 
     Set A = same-group causal pairs, set B = cross-group pairs inside the window; each set gets its
-    own softmax attention and logsumexp, joined by the Appendix C merge formula.  With
+    own softmax attention and logsumexp, joined by the Appendix D merge formula.  With
     ``double_count=True`` set B is replaced by *all* local pairs (the overlapping decomposition the
     paper rejects), which counts same-group local pairs twice.
     q_bits/k_bits/v_bits uint16 [n, D].  Returns (O [n, D], lse [n]).

@@ -328,7 +328,6 @@ int focus_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k, foc
         return rc;
     if (!lse) return fail(FOCUS_ERR_INVALID_ARG, "lse is NULL");
     if (tiles_ws && (!mq || !mk)) return fail(FOCUS_ERR_INVALID_ARG, "mq/mk are required with a tiles workspace");
-    if ((rc = require_sm100())) return rc;
     AttnArgs a;
     a.s = *shape;
     a.q = q; a.k = k; a.v = v; a.o = o;
@@ -339,6 +338,11 @@ int focus_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k, foc
     a.scale = shape->scale > 0.f ? shape->scale : 1.0f / sqrtf((float)shape->D);
     memset(&a.L, 0, sizeof a.L);
     if (tiles_ws && (rc = layout_of(shape, layout, &a.L))) return rc;
+    // The sorted layouts can refuse on the device (more mask values in a head than the class table holds) and then leave
+    // O / lse unwritten: the only way to learn of it is the status word, so it is required there.
+    if (tiles_ws && a.L.layout != FOCUS_LAYOUT_ORIGINAL && !dev_status)
+        return fail(FOCUS_ERR_INVALID_ARG, "dev_status is required with a sorted layout (it reports a refused class table)");
+    if ((rc = require_sm100())) return rc;
     return launch_attn_sm100(a, (cudaStream_t)stream);
 }
 

@@ -1,5 +1,5 @@
 // Pieces shared by the attention kernels (one CTA per SM, and one CTA pair per two SMs): launch parameters, the walk over
-// the key tiles an item visits, the per-tile keep bitmaps of the Focus mask (paper Appendix C, first equation), the order
+// the key tiles an item visits, the per-tile keep bitmaps of the Focus mask (paper Appendix D, first equation), the order
 // in which items are handed out.
 #pragma once
 
@@ -270,7 +270,8 @@ __device__ __forceinline__ void build_tile_mask_sorted(TileMask& tm, int w, cons
     const int k_first = __ldg(kpos), k_last = __ldg(kpos + 127);
     tm.all_masked = wmax < 0 || k_first > wmax;
     const bool none = !share && !window_ok;
-    const bool any_none = __any_sync(0xffffffffu, none);        // (every lane takes part: no short-circuit before it)
+    // (window_ok is the same for the whole grid, so the vote is skipped or taken by every lane alike)
+    const bool any_none = !window_ok && __any_sync(0xffffffffu, none);
     const bool need_causal = k_last > wmin;
     const bool need_window = !share && ((long long)wmax - k_first > w);
     tm.masked = need_causal || need_window || any_none;

@@ -1,5 +1,5 @@
 // focus_attn_fwd for sm_100a: persistent, warp-specialised attention forward over the attended
-// pairs of the Focus mask (paper Sec. 2 and Appendix C, first equation).
+// pairs of the Focus mask (paper Sec. 2 and Appendix D, first equation).
 //
 // One CTA per SM works through (head, 256-query block) items.  Per item, two 128-row query tiles
 // share every key/value tile that is fetched:

@@ -1,5 +1,5 @@
 // focus_decode_step: one new query token per head against the cached keys and values, under the
-// same rule as the forward pass (paper Sec. 2 "Efficiency at inference", Appendix C first equation):
+// same rule as the forward pass (paper Sec. 2 "Efficiency at inference", Appendix D first equation):
 // the new token at position n-1 attends key j when n-1-j <= w or its groups meet the key's groups.
 // This is the generation use of the method (the paper evaluates generation but gives no procedure).
 //

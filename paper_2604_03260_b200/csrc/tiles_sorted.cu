@@ -471,7 +471,7 @@ int launch_build_tiles_sorted(const focus_shape* s, const uint32_t* mq, const ui
 }
 
 // ---- FOCUS_LAYOUT_SORTED_LOCAL: the two partial results (sharing pairs from the class-sorted pass, window-only pairs
-// from the pass in token order) cover disjoint sets of pairs and join through their logsumexps (paper Appendix C).
+// from the pass in token order) cover disjoint sets of pairs and join through their logsumexps (paper Appendix D).
 
 __global__ void __launch_bounds__(256) fill_f32_kernel(float* __restrict__ x, size_t count, float v) {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;

@@ -86,6 +86,7 @@ def test_null_and_misaligned_arguments_never_reach_the_device():
         assert L.focus_attn_fwd(ctypes.byref(s), bad, t_ok, t_ok, None, None, None, 0, t_ok, 4096, None, None) == -1
     assert L.focus_attn_fwd(ctypes.byref(s), t_ok, t_ok, t_ok, None, None, None, 0, t_ok, None, None, None) == -1
     assert L.focus_attn_fwd(ctypes.byref(s), t_ok, t_ok, t_ok, None, None, 4096, 0, t_ok, 4096, None, None) == -1
+    assert L.focus_attn_fwd(ctypes.byref(s), t_ok, t_ok, t_ok, 4096, 4096, 4096, 1, t_ok, 4096, None, None) == -1   # sorted layout without a status word
     assert L.focus_count_kept(ctypes.byref(s), None, 4096, 4096, None) == -1
 
 

@@ -1,6 +1,6 @@
 """FOCUS_LAYOUT_GROUP_MAJOR: queries sorted by class, keys laid out as K lists (a key once per group it belongs to), a
 sharing pair attended under its lowest shared group, window-only pairs from the pass in token order, merged through
-the logsumexps (paper Sec. 2 "Sort tokens by group"; Sec. 3.6 top-k membership; Appendix C "Disjoint decomposition"
+the logsumexps (paper Sec. 2 "Sort tokens by group"; Sec. 3.6 top-k membership; Appendix D "Disjoint decomposition"
 and "Merge").  The structures against the oracle's definition, the attention against the fp64 oracle of the rule."""
 import numpy as np
 import pytest

@@ -1,5 +1,5 @@
 """FOCUS_LAYOUT_SORTED_LOCAL: the class-sorted pass over the pairs that share a group, the pass in token order over
-the pairs kept by the window alone, and their logsumexp merge (paper Appendix C) -- against the fp64 oracle of the
+the pairs kept by the window alone, and their logsumexp merge (paper Appendix D) -- against the fp64 oracle of the
 whole rule, with the tolerances of the other layouts."""
 import numpy as np
 import pytest

@@ -187,7 +187,7 @@ def test_softcap_closed_form_and_limit():
 
 
 def test_two_set_merge_matches_and_double_count_fails():
-    """Appendix C: sets A (same-group causal) and B (cross-group local) merged through their
+    """Appendix D: sets A (same-group causal) and B (cross-group local) merged through their
     logsumexps equal the masked definition (the paper reports cosine similarity 1.0000); the
     overlapping same-group + all-local split double counts and must NOT match."""
     rng = np.random.default_rng(11)
