@@ -160,8 +160,13 @@ FOCUS_API const char* focus_last_error(void);
  *   centroids   device, fp32 [Hkv, K, D] contiguous; need not be unit length
  *   masks_out   device, uint32 [batch*H, n]
  *   near_ties   device, nullable: *near_ties is incremented (not reset) by the number of vectors whose
- *               margin cos(topk-th) - cos((topk+1)-th), computed in fp32, is below near_tie_eps
- * Arithmetic is fp32 on the exact bf16 values.
+ *               margin cos(topk-th) - cos((topk+1)-th), computed in fp32, is below near_tie_eps.
+ *               Bit 63 of the word is the kernel's fault flag: it is set when a bounded wait inside the
+ *               kernel ran out (4 s) or the kernel found its shared memory misplaced; the masks of the
+ *               blocks concerned are then not written.  A caller that passes NULL gets no such report.
+ * Arithmetic: the dot products run on the tensor cores with each fp32 centroid split into three bf16
+ * terms, so every product with a bf16 vector element is exact and the sums are fp32; |x|, |c_g| and the
+ * selection are plain fp32.  Scores agree with the exactly rounded cosine to about 1e-6.
  */
 FOCUS_API int focus_assign(const focus_shape* shape, focus_tensor x, int32_t H, const float* centroids,
                  uint32_t* masks_out, unsigned long long* near_ties, float near_tie_eps, void* stream);

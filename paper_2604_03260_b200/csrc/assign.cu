@@ -1,131 +1,313 @@
 // focus_assign: cosine of every head vector with the K centroids of its KV head, top-k membership
-// mask out (paper Eq. 1 + the top-k rule of Sec. 3.6).  HBM-bound: each vector is read once with
-// 16-byte loads by the one thread that owns the token; the centroids of the block's KV head sit in
-// shared memory.
+// mask out (paper Eq. 1 + the top-k rule of Sec. 3.6).  HBM-bound: 2 D bytes read and 4 written per vector.
+//
+// The tiles of 128 vectors, numbered head by head, are dealt out as one contiguous range per block, a few blocks
+// per SM and all of them resident, so the launch is a single wave of equal shares.  The rows of a tile go to
+// shared memory with coalesced asynchronous 16-byte copies, laid out as the K-major, 128-byte-swizzled operand of
+// a tcgen05 MMA, two tiles in flight; whenever its range enters a head with another centroid set the block splits
+// those centroids into three bf16 terms each (hi + mid + lo carries 24 mantissa bits, so the products with the
+// bf16 vectors sum to the fp32 dot product) as the second operand.  Per tile one thread issues the MMA chain S = X C'^T (128 x 3K, fp32, in tensor
+// memory); while it runs every thread sums the squares of its own row from shared memory; then it reads its
+// row of S, adds the three terms per group, scales by 1/(|x| |c_g|), selects the top-k groups and writes its
+// mask word, while the copies of the tile after next are already under way.
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace focus {
 
-constexpr int ASSIGN_THREADS = 128;   // one thread per token: 128 tokens of one head per block
+using namespace ptx;
 
-// Thread = token.  The block copies its 128 rows into shared memory with coalesced asynchronous 16-byte
-// copies (all in flight at once); each thread then reads its own row, accumulates |x|^2 and the K dot products
-// against the centroids held in shared memory (every lane reads the same centroid words: broadcast,
-// no bank conflicts), then selects its top-k groups and writes its mask word (coalesced).
+constexpr int ASSIGN_THREADS = 128;   // one thread per vector = one lane of tensor memory
+
+template <int D, int KMAX>
+struct AssignCfg {
+    static constexpr int NCOLS = (3 * KMAX + 15) / 16 * 16;             // rows of C' = columns of S
+    static constexpr uint32_t SUB_BYTES = 128 * 128;                     // 128 vectors x 64 dimensions
+    static constexpr uint32_t TILE_BYTES = SUB_BYTES * (D / 64);
+    static constexpr uint32_t CSUB_BYTES = NCOLS * 128;                  // NCOLS rows x 64 dimensions
+    static constexpr uint32_t C_BYTES = CSUB_BYTES * (D / 64);
+    static constexpr uint32_t TMEM_COLS2 = 2 * NCOLS <= 32 ? 32 : (2 * NCOLS <= 64 ? 64 : (2 * NCOLS <= 128 ? 128 : 256));   // two S buffers
+    static constexpr uint32_t SMEM_BYTES = 2 * TILE_BYTES + C_BYTES + 256;
+    static_assert(C_BYTES % 1024 == 0, "the vector tile and the centroid operand both start on a swizzle atom");
+};
+
+struct AssignCtl {
+    uint64_t s_full[2];               // the MMA chain of the tile in buffer 0 / 1 has completed
+    uint32_t tmem_base;
+    int fault;
+    float cn2[32];                    // |c_g|^2, then 1/|c_g|
+};
+
+// byte offset of element (row, col) inside a K-major tile of `rows` rows stored as 64-column sub-tiles with the
+// 128-byte swizzle the MMA descriptors use (16-byte chunk index XOR row mod 8)
+__device__ __forceinline__ uint32_t sw128_offset(int row, int col, int rows) {
+    const int sub = col >> 6, c = col & 63;
+    return (uint32_t)(sub * rows * 128 + row * 128 + ((((c * 2) >> 4) ^ (row & 7)) << 4) + ((c * 2) & 15));
+}
+
 template <int D, int KMAX>
 __global__ void __launch_bounds__(ASSIGN_THREADS)
 assign_kernel(const __nv_bfloat16* __restrict__ x, int64_t stride_b, int64_t stride_h, int64_t stride_n,
-              int H, int G, int n, int K, int topk, const float* __restrict__ C,
+              int H, int G, int n, int K, int topk, int ntile, int share, int extra, const float* __restrict__ C,
               uint32_t* __restrict__ masks, unsigned long long* near_ties, float eps) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    float* cs = reinterpret_cast<float*>(smem_raw);            // [KMAX][D], rows >= K are zero
-    float* cinv = cs + KMAX * D;                               // [KMAX] 1/|c_g|
-    unsigned char* tile = reinterpret_cast<unsigned char*>(cinv + KMAX);   // [ASSIGN_THREADS] rows of 2D + 16 bytes
-    constexpr int ROWB = 2 * D + 16;                           // padded row: conflict-free 16-byte reads per token
+    using Cfg = AssignCfg<D, KMAX>;
+    extern __shared__ __align__(1024) unsigned char sm[];
+    const uint32_t base = smem_u32(sm);
+    const uint32_t sx = base;                                  // two vector tiles
+    const uint32_t sc = base + 2 * Cfg::TILE_BYTES;            // centroid operand C'
+    unsigned char* const cprime = sm + 2 * Cfg::TILE_BYTES;
+    AssignCtl* const ctl = reinterpret_cast<AssignCtl*>(sm + 2 * Cfg::TILE_BYTES + Cfg::C_BYTES);
+    constexpr int CPR = D / 8;                                 // 16-byte chunks per row
+    constexpr int RSTEP = ASSIGN_THREADS / CPR;                // rows covered by one copy per thread
 
-    const int bh = blockIdx.y;
-    const int b = bh / H, h = bh % H;
-    const int hk = h / G;
-    const int tok = blockIdx.x * ASSIGN_THREADS + threadIdx.x;
+    // block i takes `share` items, the first `extra` blocks one more: items item0 .. item0 + T - 1 of the list
+    // (batch * head, tile), tile fastest
+    const int item0 = blockIdx.x * share + min((int)blockIdx.x, extra);
+    const int T = share + ((int)blockIdx.x < extra ? 1 : 0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const bool in = tok < n;
+    // the swizzle is a function of the shared-memory address: a base off the 1024-byte grid would scramble both
+    // operands, so such a block reports a fault and computes nothing
+    const bool aligned = (base & 1023u) == 0;
 
-    // the block's rows first, as coalesced asynchronous 16-byte copies into shared memory (consecutive
-    // threads copy consecutive chunks of a row); they overlap the staging of the centroids
-    {
-        const __nv_bfloat16* xh = x + (size_t)b * stride_b + (size_t)h * stride_h;
-        const int tok0 = blockIdx.x * ASSIGN_THREADS;
+    // ---- copies of one tile: consecutive threads copy consecutive chunks of a row, a thread's next copy is RSTEP rows
+    // further down; rows past n are not copied (what their lanes compute is never written or counted).  Every call
+    // commits one group, empty when the tile does not exist.
+    const int r0 = threadIdx.x / CPR, cc = threadIdx.x % CPR;
+    const __nv_bfloat16* const xrow0 = x + (size_t)r0 * stride_n + cc * 8;
+    const size_t step = (size_t)RSTEP * stride_n;
+    const uint32_t dst0 = sx + (cc >> 3) * Cfg::SUB_BYTES + r0 * 128;
+    auto copy_tile = [&](int t) {
+        if (t < T) {
+            const int bh = (item0 + t) / ntile, tok0 = ((item0 + t) % ntile) * 128;
+            const __nv_bfloat16* src = xrow0 + (size_t)(bh / H) * stride_b + (size_t)(bh % H) * stride_h + (size_t)tok0 * stride_n;
+            const int left = n - tok0 - r0;                    // copy i is in range iff i * RSTEP < left
+            const uint32_t dstb = dst0 + (t & 1) * Cfg::TILE_BYTES;
 #pragma unroll
-        for (int i = 0; i < D / 8; ++i) {
-            const int q = i * ASSIGN_THREADS + threadIdx.x;
-            const int r = q / (D / 8), c = q % (D / 8);
-            if (tok0 + r < n) {
-                const uint32_t dst = (uint32_t)__cvta_generic_to_shared(tile + r * ROWB + c * 16);
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(xh + (size_t)(tok0 + r) * stride_n + c * 8)
-                             : "memory");
+            for (int i = 0; i < ASSIGN_THREADS / RSTEP; ++i) {
+                const uint32_t dst = dstb + i * RSTEP * 128 + ((((uint32_t)cc & 7u) ^ ((uint32_t)(r0 + (i * RSTEP) % 8) & 7u)) << 4);
+                if (i * RSTEP < left) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+                src += step;
             }
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    copy_tile(0);
+    copy_tile(1);
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), Cfg::TMEM_COLS2);
+        tmem_relinquish();
     }
-
-    for (int i = threadIdx.x; i < KMAX * D; i += ASSIGN_THREADS) cs[i] = i < K * D ? C[(size_t)hk * K * D + i] : 0.f;
+    if (threadIdx.x == 32) {
+        mbar_init(smem_u32(&ctl->s_full[0]), 1);
+        mbar_init(smem_u32(&ctl->s_full[1]), 1);
+        fence_mbar_init();
+        ctl->fault = 0;
+    }
     __syncthreads();
-    for (int g = warp; g < KMAX; g += ASSIGN_THREADS / 32) {      // one warp per centroid norm
-        float s = 0.f;
-        for (int d = lane; d < D; d += 32) s = fmaf(cs[g * D + d], cs[g * D + d], s);
+
+    // ---- C': the centroids of KV head hk, each split into hi + mid + lo (rows g, KMAX + g, 2 KMAX + g); the rest zero.
+    // Called by the whole block between tiles: every MMA that read the previous C' has completed, and the first
+    // barrier keeps the previous norms until every thread has used them.
+    auto build_centroids = [&](int hk) {
+        __syncthreads();
+        if (threadIdx.x < 32) ctl->cn2[threadIdx.x] = 0.f;
+        __syncthreads();
+        const float* Ch = C + (size_t)hk * K * D;
 #pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-        if (lane == 0) cinv[g] = s > 0.f ? rsqrtf(s) : 0.f;
+        for (int j = 0; j < KMAX * D / ASSIGN_THREADS; ++j) {
+            const int e = j * ASSIGN_THREADS + threadIdx.x;
+            const int g = e / D, d = e % D;                     // g is the same for the 32 lanes of a warp (D >= 64)
+            float v = g < K ? __ldg(Ch + e) : 0.f;
+            float s = v * v;
+            const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+            v -= __bfloat162float(hi);
+            const __nv_bfloat16 mid = __float2bfloat16_rn(v);
+            v -= __bfloat162float(mid);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(v);
+            *reinterpret_cast<__nv_bfloat16*>(cprime + sw128_offset(g, d, Cfg::NCOLS)) = hi;
+            *reinterpret_cast<__nv_bfloat16*>(cprime + sw128_offset(KMAX + g, d, Cfg::NCOLS)) = mid;
+            *reinterpret_cast<__nv_bfloat16*>(cprime + sw128_offset(2 * KMAX + g, d, Cfg::NCOLS)) = lo;
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+            if (lane == 0) atomicAdd(&ctl->cn2[g], s);
+        }
+        constexpr int ZROWS = Cfg::NCOLS - 3 * KMAX;           // whole rows, so the swizzle does not matter for them
+        if constexpr (ZROWS > 0) {
+            for (int i = threadIdx.x; i < ZROWS * (D / 64) * 8; i += ASSIGN_THREADS) {
+                const int sub = i / (ZROWS * 8), rem = i % (ZROWS * 8);
+                *reinterpret_cast<uint4*>(cprime + sub * Cfg::CSUB_BYTES + (3 * KMAX) * 128 + rem * 16) = make_uint4(0, 0, 0, 0);
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x < KMAX) {
+            const float s = ctl->cn2[threadIdx.x];
+            ctl->cn2[threadIdx.x] = s > 0.f ? rsqrtf(s) : 0.f;  // read by everyone after the tile's first barrier
+        }
+    };
+
+    bool ok = aligned;
+    uint32_t tmem = 0;
+    unsigned int near_votes = 0;
+    int cur_hk = -1;
+    for (int t = 0; t < T; ++t) {
+        const int buf = t & 1;
+        const int bh = (item0 + t) / ntile, tile = (item0 + t) % ntile;
+        const int hk = (bh % H) / G;
+        if (hk != cur_hk) {
+            build_centroids(hk);
+            cur_hk = hk;
+        }
+        asm volatile("cp.async.wait_group 1;" ::: "memory");   // this thread's copies of tile t have landed
+        fence_proxy_async_smem();                              // generic-proxy writes before the MMA's async-proxy reads
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        tmem = ctl->tmem_base;
+        if (warp == 0) {
+            if (aligned && elect_one()) {
+                constexpr uint32_t IDESC = idesc_bf16(128, Cfg::NCOLS, 0, 0);
+                const uint64_t xd = smem_desc_sw128(sx + buf * Cfg::TILE_BYTES, 16, 1024);
+                const uint64_t cd = smem_desc_sw128(sc, 16, 1024);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)
+                    umma_ss(tmem + buf * Cfg::NCOLS, xd + (uint64_t)(((ks / 4) * Cfg::SUB_BYTES + (ks % 4) * 32) >> 4),
+                            cd + (uint64_t)(((ks / 4) * Cfg::CSUB_BYTES + (ks % 4) * 32) >> 4), IDESC, ks > 0);
+                umma_commit(smem_u32(&ctl->s_full[buf]));
+            }
+            __syncwarp();
+        }
+        // ---- |x|^2 of the thread's own row while the MMAs run (packed fp32 pairs)
+        float xx;
+        {
+            const unsigned char* row = sm + buf * Cfg::TILE_BYTES + threadIdx.x * 128;
+            const uint32_t sw = (threadIdx.x & 7u) << 4;
+            float2 a0 = make_float2(0.f, 0.f), a1 = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int v = 0; v < CPR; ++v) {
+                const uint4 rv = *reinterpret_cast<const uint4*>(row + (v >> 3) * Cfg::SUB_BYTES + ((((uint32_t)v & 7u) << 4) ^ sw));
+                const float2 v0 = make_float2(__uint_as_float(rv.x << 16), __uint_as_float(rv.x & 0xffff0000u));
+                const float2 v1 = make_float2(__uint_as_float(rv.y << 16), __uint_as_float(rv.y & 0xffff0000u));
+                const float2 v2 = make_float2(__uint_as_float(rv.z << 16), __uint_as_float(rv.z & 0xffff0000u));
+                const float2 v3 = make_float2(__uint_as_float(rv.w << 16), __uint_as_float(rv.w & 0xffff0000u));
+                a0 = __ffma2_rn(v0, v0, a0); a1 = __ffma2_rn(v1, v1, a1);
+                a0 = __ffma2_rn(v2, v2, a0); a1 = __ffma2_rn(v3, v3, a1);
+            }
+            xx = (a0.x + a0.y) + (a1.x + a1.y);
+        }
+        if (ok && !mbar_wait(smem_u32(&ctl->s_full[buf]), (uint32_t)((t >> 1) & 1))) {
+            ok = false;
+            ctl->fault = 1;
+        }
+        tc_fence_after();
+        float sc3[Cfg::NCOLS];
+        if (ok) {
+#pragma unroll
+            for (int c = 0; c < Cfg::NCOLS / 16; ++c) {
+                uint32_t v[16];
+                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + buf * Cfg::NCOLS + c * 16, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 16; ++e) sc3[c * 16 + e] = __uint_as_float(v[e]);
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < Cfg::NCOLS; ++e) sc3[e] = 0.f;
+        }
+        tc_fence_before();
+        __syncthreads();                                       // the tile's buffer is free: its MMAs and every row sum are done
+        copy_tile(t + 2);
+
+        const int tok = tile * 128 + threadIdx.x;
+        const bool in = tok < n;
+        const float xinv = xx > 0.f ? rsqrtf(xx) : 0.f;
+        float cosv[KMAX];
+#pragma unroll
+        for (int g = 0; g < KMAX; ++g) cosv[g] = ((sc3[2 * KMAX + g] + sc3[KMAX + g]) + sc3[g]) * ctl->cn2[g] * xinv;
+        uint32_t taken = 0;
+        float last = 0.f, next = 0.f;
+        if constexpr (KMAX <= 8) {
+            // rank of every group among the K (how many beat it; the lower index wins an exact tie): the
+            // groups of rank < topk are taken, the margin is between rank topk-1 and rank topk
+            int rank[KMAX];
+#pragma unroll
+            for (int g = 0; g < KMAX; ++g) {
+                rank[g] = 0;
+                if (g >= K) cosv[g] = -INFINITY;
+            }
+#pragma unroll
+            for (int a = 0; a < KMAX; ++a)
+#pragma unroll
+                for (int c = a + 1; c < KMAX; ++c) {
+                    const bool a_first = !(cosv[c] > cosv[a]);
+                    rank[c] += a_first ? 1 : 0;
+                    rank[a] += a_first ? 0 : 1;
+                }
+            const int kk = topk < K ? topk : K;
+#pragma unroll
+            for (int g = 0; g < KMAX; ++g) {
+                if (g < K && rank[g] < kk) taken |= 1u << g;
+                if (rank[g] == kk - 1) last = cosv[g];
+                if (rank[g] == kk) next = cosv[g];
+            }
+        } else {
+            // topk picks, then one more to measure the margin; strict '>' keeps the lowest index on ties
+            for (int it = 0; it <= topk && it < K; ++it) {
+                float best = -INFINITY;
+                int bi = 0;
+#pragma unroll
+                for (int g = 0; g < KMAX; ++g) {
+                    const bool better = g < K && !((taken >> g) & 1u) && (cosv[g] > best || best == -INFINITY);
+                    if (better) { best = cosv[g]; bi = g; }
+                }
+                if (it < topk) { taken |= 1u << bi; last = best; }
+                else next = best;
+            }
+        }
+        if (in && ok) masks[(size_t)bh * n + tok] = taken;
+        if (near_ties) near_votes += __popc(__ballot_sync(0xffffffffu, ok && in && topk < K && (last - next) < eps));
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (near_ties && lane == 0 && near_votes) atomicAdd(near_ties, (unsigned long long)near_votes);
     __syncthreads();
-
-    // packed fp32 pairs: even elements accumulate in .x, odd elements in .y
-    float2 xx2 = make_float2(0.f, 0.f);
-    float2 dot2[KMAX];
-#pragma unroll
-    for (int g = 0; g < KMAX; ++g) dot2[g] = make_float2(0.f, 0.f);
-#pragma unroll
-    for (int v = 0; v < D / 8; ++v) {
-        const uint4 rv = in ? *reinterpret_cast<const uint4*>(tile + threadIdx.x * ROWB + v * 16) : make_uint4(0, 0, 0, 0);
-        const uint32_t wds[4] = {rv.x, rv.y, rv.z, rv.w};
-        float2 xv[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) xv[e] = make_float2(__uint_as_float(wds[e] << 16), __uint_as_float(wds[e] & 0xffff0000u));
-#pragma unroll
-        for (int e = 0; e < 4; ++e) xx2 = __ffma2_rn(xv[e], xv[e], xx2);
-#pragma unroll
-        for (int g = 0; g < KMAX; ++g) {
-            const float4 c0 = *reinterpret_cast<const float4*>(cs + g * D + v * 8);
-            const float4 c1 = *reinterpret_cast<const float4*>(cs + g * D + v * 8 + 4);
-            float2 sacc = dot2[g];
-            sacc = __ffma2_rn(xv[0], make_float2(c0.x, c0.y), sacc);
-            sacc = __ffma2_rn(xv[1], make_float2(c0.z, c0.w), sacc);
-            sacc = __ffma2_rn(xv[2], make_float2(c1.x, c1.y), sacc);
-            sacc = __ffma2_rn(xv[3], make_float2(c1.z, c1.w), sacc);
-            dot2[g] = sacc;
+    if (warp == 0) {
+        if (ctl->fault || !aligned) {
+            if (lane == 0 && near_ties) atomicOr(near_ties, 1ull << 63);
+            const uint64_t t0 = globaltimer_ns();
+            while (globaltimer_ns() - t0 < 20000ull) { }       // MMAs already issued finish before the columns go back
         }
-    }
-    const float xx = xx2.x + xx2.y;
-    float dot[KMAX];
-#pragma unroll
-    for (int g = 0; g < KMAX; ++g) dot[g] = dot2[g].x + dot2[g].y;
-    const float xinv = xx > 0.f ? rsqrtf(xx) : 0.f;
-    float cosv[KMAX];
-#pragma unroll
-    for (int g = 0; g < KMAX; ++g) cosv[g] = dot[g] * cinv[g] * xinv;
-    uint32_t taken = 0;
-    float last = 0.f, next = 0.f;
-    // topk picks, then one more to measure the margin; strict '>' keeps the lowest index on ties
-    for (int it = 0; it <= topk && it < K; ++it) {
-        float best = -INFINITY;
-        int bi = 0;
-#pragma unroll
-        for (int g = 0; g < KMAX; ++g) {
-            const bool ok = g < K && !((taken >> g) & 1u) && (cosv[g] > best || best == -INFINITY);
-            if (ok) { best = cosv[g]; bi = g; }
-        }
-        if (it < topk) { taken |= 1u << bi; last = best; }
-        else next = best;
-    }
-    if (in) masks[(size_t)bh * n + tok] = taken;
-    if (near_ties) {
-        const unsigned int near = __ballot_sync(0xffffffffu, in && topk < K && (last - next) < eps);
-        if (lane == 0 && near) atomicAdd(near_ties, (unsigned long long)__popc(near));
+        tmem_dealloc(ctl->tmem_base, Cfg::TMEM_COLS2);
     }
 }
 
 template <int D, int KMAX>
 static int launch_one(const focus_shape* s, const focus_tensor& x, int H, const float* C, uint32_t* masks,
                       unsigned long long* near_ties, float eps, cudaStream_t st) {
-    const size_t smem = (size_t)(KMAX * D + KMAX) * sizeof(float) + (size_t)ASSIGN_THREADS * (2 * D + 16);
+    using Cfg = AssignCfg<D, KMAX>;
     auto kern = assign_kernel<D, KMAX>;
-    int rc = check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
+    int rc = check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM_BYTES),
                         "cudaFuncSetAttribute(assign)");
     if (rc) return rc;
-    dim3 grid(cdiv(s->n, ASSIGN_THREADS), s->batch * H);
-    kern<<<grid, ASSIGN_THREADS, smem, st>>>(reinterpret_cast<const __nv_bfloat16*>(x.ptr), x.stride_b, x.stride_h,
-                                              x.stride_n, H, H / s->Hkv, s->n, s->K, s->topk, C, masks, near_ties, eps);
+    if ((rc = check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100), "cudaFuncSetAttribute(assign)"))) return rc;
+    // one resident wave: as many blocks as fit on the device at once (fewer when there are fewer tiles).  Blocks of
+    // 128 threads per SM: by shared memory (227 KB, 1 KB reserved per block), by the 512 columns of tensor memory, and
+    // at most 4 (64 K registers, up to 128 per thread)
+    int dev = 0, sms = 0;
+    if ((rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice"))) return rc;
+    if ((rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "cudaDeviceGetAttribute"))) return rc;
+    int per_sm = (int)(227 * 1024 / (Cfg::SMEM_BYTES + 1024));
+    if (per_sm > (int)(512 / Cfg::TMEM_COLS2)) per_sm = (int)(512 / Cfg::TMEM_COLS2);
+    if (per_sm > 4) per_sm = 4;
+    if (per_sm < 1) per_sm = 1;
+    const long long resident = (long long)sms * per_sm;
+    const int ntile = cdiv(s->n, 128);
+    const long long nitems = (long long)s->batch * H * ntile;
+    if (nitems > 0x7fffffffll) return fail(FOCUS_ERR_UNSUPPORTED, "focus_assign: %lld tiles of 128 vectors exceed 2^31 - 1", nitems);
+    if (nitems == 0) return 0;
+    const int nblocks = (int)(nitems < resident ? nitems : resident);
+    const int share = (int)(nitems / nblocks), extra = (int)(nitems % nblocks);
+    kern<<<nblocks, ASSIGN_THREADS, Cfg::SMEM_BYTES, st>>>(reinterpret_cast<const __nv_bfloat16*>(x.ptr), x.stride_b, x.stride_h,
+                                                           x.stride_n, H, H / s->Hkv, s->n, s->K, s->topk, ntile, share, extra, C, masks,
+                                                           near_ties, eps);
     return check_cuda(cudaGetLastError(), "assign kernel launch");
 }
 

@@ -18,7 +18,9 @@ def gpu_assign(wl, X, C, H):
     near = torch.zeros(1, dtype=torch.int64, device="cuda")
     fb.focus_assign(shape, X, H, C, masks, near, 1e-5)
     torch.cuda.synchronize()
-    return masks, int(near.item())
+    count = int(near.item()) & (2 ** 64 - 1)
+    assert count >> 63 == 0, "focus_assign set its fault flag (bit 63 of the near-tie word)"
+    return masks, count
 
 
 def gpu_tiles(wl, mq, mk, layout=0):
