@@ -10,7 +10,7 @@
 // memory); while it runs every thread sums the squares of its own row from shared memory; then it reads its
 // row of S, adds the three terms per group, scales by 1/(|x| |c_g|), selects the top-k groups and writes its
 // mask word, while the copies of the tile after next are already under way.
-#include "common.cuh"
+#include "assign_common.cuh"
 #include "sm100_ptx.cuh"
 
 namespace focus {
@@ -37,13 +37,6 @@ struct AssignCtl {
     int fault;
     float cn2[32];                    // |c_g|^2, then 1/|c_g|
 };
-
-// byte offset of element (row, col) inside a K-major tile of `rows` rows stored as 64-column sub-tiles with the
-// 128-byte swizzle the MMA descriptors use (16-byte chunk index XOR row mod 8)
-__device__ __forceinline__ uint32_t sw128_offset(int row, int col, int rows) {
-    const int sub = col >> 6, c = col & 63;
-    return (uint32_t)(sub * rows * 128 + row * 128 + ((((c * 2) >> 4) ^ (row & 7)) << 4) + ((c * 2) & 15));
-}
 
 template <int D, int KMAX>
 __global__ void __launch_bounds__(ASSIGN_THREADS)
@@ -119,11 +112,8 @@ assign_kernel(const __nv_bfloat16* __restrict__ x, int64_t stride_b, int64_t str
             const int g = e / D, d = e % D;                     // g is the same for the 32 lanes of a warp (D >= 64)
             float v = g < K ? __ldg(Ch + e) : 0.f;
             float s = v * v;
-            const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-            v -= __bfloat162float(hi);
-            const __nv_bfloat16 mid = __float2bfloat16_rn(v);
-            v -= __bfloat162float(mid);
-            const __nv_bfloat16 lo = __float2bfloat16_rn(v);
+            __nv_bfloat16 hi, mid, lo;
+            split3_bf16(v, hi, mid, lo);
             *reinterpret_cast<__nv_bfloat16*>(cprime + sw128_offset(g, d, Cfg::NCOLS)) = hi;
             *reinterpret_cast<__nv_bfloat16*>(cprime + sw128_offset(KMAX + g, d, Cfg::NCOLS)) = mid;
             *reinterpret_cast<__nv_bfloat16*>(cprime + sw128_offset(2 * KMAX + g, d, Cfg::NCOLS)) = lo;
@@ -223,46 +213,8 @@ assign_kernel(const __nv_bfloat16* __restrict__ x, int64_t stride_b, int64_t str
         float cosv[KMAX];
 #pragma unroll
         for (int g = 0; g < KMAX; ++g) cosv[g] = ((sc3[2 * KMAX + g] + sc3[KMAX + g]) + sc3[g]) * ctl->cn2[g] * xinv;
-        uint32_t taken = 0;
-        float last = 0.f, next = 0.f;
-        if constexpr (KMAX <= 8) {
-            // rank of every group among the K (how many beat it; the lower index wins an exact tie): the
-            // groups of rank < topk are taken, the margin is between rank topk-1 and rank topk
-            int rank[KMAX];
-#pragma unroll
-            for (int g = 0; g < KMAX; ++g) {
-                rank[g] = 0;
-                if (g >= K) cosv[g] = -INFINITY;
-            }
-#pragma unroll
-            for (int a = 0; a < KMAX; ++a)
-#pragma unroll
-                for (int c = a + 1; c < KMAX; ++c) {
-                    const bool a_first = !(cosv[c] > cosv[a]);
-                    rank[c] += a_first ? 1 : 0;
-                    rank[a] += a_first ? 0 : 1;
-                }
-            const int kk = topk < K ? topk : K;
-#pragma unroll
-            for (int g = 0; g < KMAX; ++g) {
-                if (g < K && rank[g] < kk) taken |= 1u << g;
-                if (rank[g] == kk - 1) last = cosv[g];
-                if (rank[g] == kk) next = cosv[g];
-            }
-        } else {
-            // topk picks, then one more to measure the margin; strict '>' keeps the lowest index on ties
-            for (int it = 0; it <= topk && it < K; ++it) {
-                float best = -INFINITY;
-                int bi = 0;
-#pragma unroll
-                for (int g = 0; g < KMAX; ++g) {
-                    const bool better = g < K && !((taken >> g) & 1u) && (cosv[g] > best || best == -INFINITY);
-                    if (better) { best = cosv[g]; bi = g; }
-                }
-                if (it < topk) { taken |= 1u << bi; last = best; }
-                else next = best;
-            }
-        }
+        float last, next;
+        const uint32_t taken = select_topk<KMAX>(cosv, K, topk, last, next);
         if (in && ok) masks[(size_t)bh * n + tok] = taken;
         if (near_ties) near_votes += __popc(__ballot_sync(0xffffffffu, ok && in && topk < K && (last - next) < eps));
     }

@@ -4,15 +4,44 @@
 //
 // W_g^T h . C_g = h . (W_g C_g), so the projection and the centroids fold into K vectors of length d
 // (a small kernel, once per call); scoring then reads each hidden state exactly once, which makes the
-// pass HBM-bound: 2 d bytes per token.  Thread = token; the block's rows stream through shared
-// memory in chunks of 64 elements (coalesced asynchronous 16-byte copies, two chunks in flight).
-#include "common.cuh"
+// pass HBM-bound: 2 d bytes per token.
+//
+// Scoring runs on the tensor cores.  The tiles of 128 tokens are dealt out as one contiguous range per block,
+// one resident wave of small blocks.  A block walks its tiles in chunks of 128 elements of d: the chunk of the
+// 128 rows goes to shared memory with coalesced asynchronous 16-byte copies, laid out as the K-major,
+// 128-byte-swizzled operand of a tcgen05 MMA, two chunks in flight; the same chunk of the K folded vectors is
+// split into three bf16 terms each (hi + mid + lo carries 24 mantissa bits, so the products with the bf16 hidden
+// states sum to the fp32 dot product) as the second operand.  One thread issues the MMAs of the chunk, which
+// accumulate S = H F'^T (128 x 3K, fp32) in tensor memory over the chunks of the tile; after the last chunk every
+// thread reads its row of S, adds the three terms per group and the bias, and selects (or stores the scores).
+#include "assign_common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace focus {
 
-constexpr int AH_THREADS = 64;       // tokens per block (small, so that modest sequence lengths still fill the GPU)
-constexpr int AH_CHUNK = 64;         // elements of a row per stage
-constexpr int AH_ROWB = 2 * AH_CHUNK + 16;   // padded row: conflict-free 16-byte reads per token
+using namespace ptx;
+
+constexpr int AH_THREADS = 128;      // one thread per token of the tile = one lane of tensor memory
+constexpr int AH_CHUNK = 128;        // elements of d per stage: two 64-column sub-tiles
+
+template <int KMAX>
+struct HiddenCfg {
+    static constexpr int NCOLS = (3 * KMAX + 15) / 16 * 16;             // rows of F' = columns of S
+    static constexpr uint32_t SUB_BYTES = 128 * 128;                     // 128 tokens x 64 elements
+    static constexpr uint32_t A_BYTES = 2 * SUB_BYTES;
+    static constexpr uint32_t FSUB_BYTES = NCOLS * 128;                  // NCOLS rows x 64 elements
+    static constexpr uint32_t F_BYTES = 2 * FSUB_BYTES;
+    static constexpr uint32_t STAGE_BYTES = A_BYTES + F_BYTES;
+    static constexpr uint32_t TMEM_COLS = NCOLS <= 32 ? 32 : (NCOLS <= 64 ? 64 : 128);
+    static constexpr uint32_t SMEM_BYTES = 2 * STAGE_BYTES + 256;
+    static_assert(STAGE_BYTES % 1024 == 0, "every operand starts on a swizzle atom");
+};
+
+struct HiddenCtl {
+    uint64_t mma_done[2];             // the MMAs that read stage 0 / 1 have completed
+    uint32_t tmem_base;
+    int fault;
+};
 
 // folded[g][e] = sum_j Wg[e][j] * C[g][j]
 __global__ void __launch_bounds__(256)
@@ -30,126 +59,216 @@ __global__ void __launch_bounds__(AH_THREADS)
 assign_hidden_kernel(const __nv_bfloat16* __restrict__ h, int64_t stride_b, int64_t stride_n, int n, int d, int K, int topk,
                      const float* __restrict__ folded, const float* __restrict__ bias, int Hq, int Hkv,
                      uint32_t* __restrict__ mq, uint32_t* __restrict__ mk, unsigned long long* near_ties, float eps,
-                     float* __restrict__ scores) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    unsigned char* tile = smem_raw;                                           // [2][AH_THREADS][AH_ROWB]
-    float* cs = reinterpret_cast<float*>(smem_raw + 2 * AH_THREADS * AH_ROWB);   // [2][KMAX][AH_CHUNK]
-    const int b = blockIdx.y;
-    const int tok0 = blockIdx.x * AH_THREADS;
-    const int tok = tok0 + threadIdx.x;
-    const bool in = tok < n;
-    const __nv_bfloat16* hb = h + (size_t)b * stride_b;
-    const int nchunk = (d + AH_CHUNK - 1) / AH_CHUNK;
+                     float* __restrict__ scores, int ntile, int share, int extra) {
+    using Cfg = HiddenCfg<KMAX>;
+    extern __shared__ __align__(1024) unsigned char sm[];
+    const uint32_t base = smem_u32(sm);
+    HiddenCtl* const ctl = reinterpret_cast<HiddenCtl*>(sm + 2 * Cfg::STAGE_BYTES);
+    constexpr int CPR = AH_CHUNK / 8;                          // 16-byte pieces per row of a chunk
+    constexpr int RSTEP = AH_THREADS / CPR;                    // rows covered by one copy per thread (8)
 
-    auto stage = [&](int ch, int buf) {
-        const int e0 = ch * AH_CHUNK;
-        const int vec = min(AH_CHUNK, d - e0) / 8;                            // 16-byte pieces per row in this chunk
-        for (int q = threadIdx.x; q < AH_THREADS * vec; q += AH_THREADS) {
-            const int r = q / vec, c = q % vec;
-            if (tok0 + r < n) {
-                const uint32_t dst = (uint32_t)__cvta_generic_to_shared(tile + ((size_t)buf * AH_THREADS + r) * AH_ROWB + c * 16);
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(hb + (size_t)(tok0 + r) * stride_n + e0 + c * 8)
-                             : "memory");
-            }
-        }
-        for (int q = threadIdx.x; q < KMAX * (AH_CHUNK / 4); q += AH_THREADS) {   // folded centroids of the chunk, 16 bytes each
-            const int g = q / (AH_CHUNK / 4), c = q % (AH_CHUNK / 4);
-            float* dstp = cs + ((size_t)buf * KMAX + g) * AH_CHUNK + c * 4;
-            if (g < K && e0 + c * 4 < d) {
-                const uint32_t dst = (uint32_t)__cvta_generic_to_shared(dstp);
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(folded + (size_t)g * d + e0 + c * 4) : "memory");
+    // block i takes `share` tiles, the first `extra` blocks one more: tiles item0 .. item0 + T - 1 of the list
+    // (batch, tile); its work is the T * nchunk chunks of those tiles, walked in order
+    const int item0 = blockIdx.x * share + min((int)blockIdx.x, extra);
+    const int T = share + ((int)blockIdx.x < extra ? 1 : 0);
+    const int nchunk = (d + AH_CHUNK - 1) / AH_CHUNK;
+    const int total = T * nchunk;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // the swizzle is a function of the shared-memory address: a base off the 1024-byte grid would scramble both
+    // operands, so such a block reports a fault and computes nothing
+    const bool aligned = (base & 1023u) == 0;
+
+    // ---- stage one chunk: rows by asynchronous copies (consecutive threads copy consecutive pieces of a row, a
+    // thread's next copy is 8 rows further down; rows past n are not copied: what their lanes compute is never
+    // written or counted; pieces past d are zero), folded vectors split on the way in (thread = column).  Every
+    // call commits one group, empty when the chunk does not exist.  (it, ic) = tile and chunk of the next call.
+    const int r0 = threadIdx.x / CPR, cc = threadIdx.x % CPR;
+    int it_next = 0, ic_next = 0;
+    auto stage_chunk = [&](int j) {
+        if (j < total) {
+            const int item = item0 + it_next;
+            const int b = item / ntile, tok0 = (item % ntile) * 128;
+            const int e0 = ic_next * AH_CHUNK;
+            unsigned char* const st = sm + (j & 1) * Cfg::STAGE_BYTES;
+            const uint32_t dstb = base + (j & 1) * Cfg::STAGE_BYTES + (cc >> 3) * Cfg::SUB_BYTES + r0 * 128 +
+                                  ((((uint32_t)cc & 7u) ^ ((uint32_t)r0 & 7u)) << 4);
+            if (e0 + cc * 8 < d) {
+                const __nv_bfloat16* src = h + (size_t)b * stride_b + (size_t)(tok0 + r0) * stride_n + e0 + cc * 8;
+                const size_t step = (size_t)RSTEP * stride_n;
+                const int left = n - tok0 - r0;                // copy i is in range iff i * RSTEP < left
+#pragma unroll
+                for (int i = 0; i < AH_THREADS / RSTEP; ++i) {
+                    if (i * RSTEP < left)
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dstb + i * RSTEP * 128), "l"(src) : "memory");
+                    src += step;
+                }
             } else {
-                *reinterpret_cast<float4*>(dstp) = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int i = 0; i < AH_THREADS / RSTEP; ++i)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dstb + i * RSTEP * 128), "r"(0) : "memory");
             }
+            unsigned char* const fp = st + Cfg::A_BYTES;
+            const int e = e0 + threadIdx.x;
+#pragma unroll
+            for (int g = 0; g < KMAX; ++g) {
+                const float v = (g < K && e < d) ? __ldg(folded + (size_t)g * d + e) : 0.f;
+                __nv_bfloat16 hi, mid, lo;
+                split3_bf16(v, hi, mid, lo);
+                *reinterpret_cast<__nv_bfloat16*>(fp + sw128_offset(g, threadIdx.x, Cfg::NCOLS)) = hi;
+                *reinterpret_cast<__nv_bfloat16*>(fp + sw128_offset(KMAX + g, threadIdx.x, Cfg::NCOLS)) = mid;
+                *reinterpret_cast<__nv_bfloat16*>(fp + sw128_offset(2 * KMAX + g, threadIdx.x, Cfg::NCOLS)) = lo;
+            }
+            if (++ic_next == nchunk) { ic_next = 0; ++it_next; }
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
 
-    float2 dot2[KMAX];
-#pragma unroll
-    for (int g = 0; g < KMAX; ++g) dot2[g] = make_float2(0.f, 0.f);
-    stage(0, 0);
-    for (int ch = 0; ch < nchunk; ++ch) {
-        const int buf = ch & 1;
-        if (ch + 1 < nchunk) {
-            stage(ch + 1, buf ^ 1);
-            asm volatile("cp.async.wait_group 1;" ::: "memory");
-        } else {
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-        }
-        __syncthreads();
-        const int vec = min(AH_CHUNK, d - ch * AH_CHUNK) / 8;
-        const unsigned char* row = tile + ((size_t)buf * AH_THREADS + threadIdx.x) * AH_ROWB;
-        const float* cb = cs + (size_t)buf * KMAX * AH_CHUNK;
-#pragma unroll 4
-        for (int v = 0; v < vec; ++v) {
-            const uint4 rv = in ? *reinterpret_cast<const uint4*>(row + v * 16) : make_uint4(0, 0, 0, 0);
-            const uint32_t wds[4] = {rv.x, rv.y, rv.z, rv.w};
-            float2 xv[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) xv[e] = make_float2(__uint_as_float(wds[e] << 16), __uint_as_float(wds[e] & 0xffff0000u));
-#pragma unroll
-            for (int g = 0; g < KMAX; ++g) {
-                const float4 c0 = *reinterpret_cast<const float4*>(cb + g * AH_CHUNK + v * 8);
-                const float4 c1 = *reinterpret_cast<const float4*>(cb + g * AH_CHUNK + v * 8 + 4);
-                float2 sacc = dot2[g];
-                sacc = __ffma2_rn(xv[0], make_float2(c0.x, c0.y), sacc);
-                sacc = __ffma2_rn(xv[1], make_float2(c0.z, c0.w), sacc);
-                sacc = __ffma2_rn(xv[2], make_float2(c1.x, c1.y), sacc);
-                sacc = __ffma2_rn(xv[3], make_float2(c1.z, c1.w), sacc);
-                dot2[g] = sacc;
+    // rows of F' beyond 3 KMAX stay zero in both stages (whole rows, so the swizzle does not matter for them)
+    {
+        constexpr int ZROWS = Cfg::NCOLS - 3 * KMAX;
+        if constexpr (ZROWS > 0) {
+            for (int i = threadIdx.x; i < 2 * 2 * ZROWS * 8; i += AH_THREADS) {
+                const int stg = i / (2 * ZROWS * 8), rem = i % (2 * ZROWS * 8);
+                const int sub = rem / (ZROWS * 8), q = rem % (ZROWS * 8);
+                *reinterpret_cast<uint4*>(sm + stg * Cfg::STAGE_BYTES + Cfg::A_BYTES + sub * Cfg::FSUB_BYTES + (3 * KMAX) * 128 + q * 16) =
+                    make_uint4(0, 0, 0, 0);
             }
         }
-        __syncthreads();            // the buffer is refilled two iterations later
     }
-    float score[KMAX];
+    stage_chunk(0);
+    stage_chunk(1);
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), Cfg::TMEM_COLS);
+        tmem_relinquish();
+    }
+    if (threadIdx.x == 32) {
+        mbar_init(smem_u32(&ctl->mma_done[0]), 1);
+        mbar_init(smem_u32(&ctl->mma_done[1]), 1);
+        fence_mbar_init();
+        ctl->fault = 0;
+    }
+
+    bool ok = aligned;
+    unsigned int near_votes = 0;
+    int it = 0, ic = 0;                                        // tile and chunk of iteration j
+    for (int j = 0; j < total; ++j) {
+        const int buf = j & 1;
+        asm volatile("cp.async.wait_group 1;" ::: "memory");   // this thread's copies of chunk j have landed
+        fence_proxy_async_smem();                              // generic-proxy writes before the MMA's async-proxy reads
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        const uint32_t tmem = ctl->tmem_base;
+        if (warp == 0) {
+            if (aligned && elect_one()) {
+                constexpr uint32_t IDESC = idesc_bf16(128, Cfg::NCOLS, 0, 0);
+                const uint64_t ad = smem_desc_sw128(base + buf * Cfg::STAGE_BYTES, 16, 1024);
+                const uint64_t fd = smem_desc_sw128(base + buf * Cfg::STAGE_BYTES + Cfg::A_BYTES, 16, 1024);
 #pragma unroll
-    for (int g = 0; g < KMAX; ++g) score[g] = dot2[g].x + dot2[g].y + ((bias && g < K) ? __ldg(bias + g) : 0.f);
-    if (scores) {   // the scores themselves (training-time soft assignment), rows of KMAX floats, zero beyond K
-        if (in) {
-            float4* o = reinterpret_cast<float4*>(scores + ((size_t)b * n + tok) * KMAX);
-#pragma unroll
-            for (int c = 0; c < KMAX / 4; ++c)
-                o[c] = make_float4(4 * c < K ? score[4 * c] : 0.f, 4 * c + 1 < K ? score[4 * c + 1] : 0.f,
-                                   4 * c + 2 < K ? score[4 * c + 2] : 0.f, 4 * c + 3 < K ? score[4 * c + 3] : 0.f);
+                for (int ks = 0; ks < AH_CHUNK / 16; ++ks)
+                    umma_ss(tmem, ad + (uint64_t)(((ks / 4) * Cfg::SUB_BYTES + (ks % 4) * 32) >> 4),
+                            fd + (uint64_t)(((ks / 4) * Cfg::FSUB_BYTES + (ks % 4) * 32) >> 4), IDESC, (ic > 0 || ks > 0) ? 1u : 0u);
+                umma_commit(smem_u32(&ctl->mma_done[buf]));
+            }
+            __syncwarp();
         }
-        return;
-    }
-    uint32_t taken = 0;
-    float last = 0.f, next = 0.f;
-    // topk picks, then one more to measure the margin; strict '>' keeps the lowest index on ties
-    for (int it = 0; it <= topk && it < K; ++it) {
-        float best = -INFINITY;
-        int bi = 0;
-#pragma unroll
-        for (int g = 0; g < KMAX; ++g) {
-            const bool ok = g < K && !((taken >> g) & 1u) && (score[g] > best || best == -INFINITY);
-            if (ok) { best = score[g]; bi = g; }
+        if (ok && !mbar_wait(smem_u32(&ctl->mma_done[buf]), (uint32_t)((j >> 1) & 1))) {
+            ok = false;
+            ctl->fault = 1;
         }
-        if (it < topk) { taken |= 1u << bi; last = best; }
-        else next = best;
+        const bool last_chunk = ic == nchunk - 1;
+        float sc3[Cfg::NCOLS];
+        if (last_chunk) {
+            tc_fence_after();
+            if (ok) {
+#pragma unroll
+                for (int c = 0; c < Cfg::NCOLS / 16; ++c) {
+                    uint32_t v[16];
+                    tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + c * 16, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) sc3[c * 16 + e] = __uint_as_float(v[e]);
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < Cfg::NCOLS; ++e) sc3[e] = 0.f;
+            }
+            tc_fence_before();
+        }
+        __syncthreads();                                       // the stage is free: its MMAs are done
+        stage_chunk(j + 2);
+
+        if (last_chunk) {
+            const int item = item0 + it;
+            const int b = item / ntile, tok = (item % ntile) * 128 + threadIdx.x;
+            const bool in = tok < n;
+            float score[KMAX];
+#pragma unroll
+            for (int g = 0; g < KMAX; ++g)
+                score[g] = ((sc3[2 * KMAX + g] + sc3[KMAX + g]) + sc3[g]) + ((bias && g < K) ? __ldg(bias + g) : 0.f);
+            if (scores) {   // the scores themselves (training-time soft assignment), rows of KMAX floats, zero beyond K
+                if (in && ok) {
+                    float4* o = reinterpret_cast<float4*>(scores + ((size_t)b * n + tok) * KMAX);
+#pragma unroll
+                    for (int c = 0; c < KMAX / 4; ++c)
+                        o[c] = make_float4(4 * c < K ? score[4 * c] : 0.f, 4 * c + 1 < K ? score[4 * c + 1] : 0.f,
+                                           4 * c + 2 < K ? score[4 * c + 2] : 0.f, 4 * c + 3 < K ? score[4 * c + 3] : 0.f);
+                }
+            } else {
+                float last, next;
+                const uint32_t taken = select_topk<KMAX>(score, K, topk, last, next);
+                if (in && ok) {   // every head of the layer shares the token's mask
+                    if (mq) for (int hh = 0; hh < Hq; ++hh) mq[((size_t)b * Hq + hh) * n + tok] = taken;
+                    if (mk) for (int hh = 0; hh < Hkv; ++hh) mk[((size_t)b * Hkv + hh) * n + tok] = taken;
+                }
+                if (near_ties) near_votes += __popc(__ballot_sync(0xffffffffu, ok && in && topk < K && (last - next) < eps));
+            }
+        }
+        if (++ic == nchunk) { ic = 0; ++it; }
     }
-    if (in) {   // every head of the layer shares the token's mask
-        if (mq) for (int hh = 0; hh < Hq; ++hh) mq[((size_t)b * Hq + hh) * n + tok] = taken;
-        if (mk) for (int hh = 0; hh < Hkv; ++hh) mk[((size_t)b * Hkv + hh) * n + tok] = taken;
-    }
-    if (near_ties) {
-        const unsigned int near = __ballot_sync(0xffffffffu, in && topk < K && (last - next) < eps);
-        if ((threadIdx.x & 31) == 0 && near) atomicAdd(near_ties, (unsigned long long)__popc(near));
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (near_ties && lane == 0 && near_votes) atomicAdd(near_ties, (unsigned long long)near_votes);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        if (ctl->fault || !aligned) {
+            if (lane == 0 && near_ties) atomicOr(near_ties, 1ull << 63);
+            const uint64_t t0 = globaltimer_ns();
+            while (globaltimer_ns() - t0 < 20000ull) { }       // MMAs already issued finish before the columns go back
+        }
+        tmem_dealloc(ctl->tmem_base, Cfg::TMEM_COLS);
     }
 }
 
 template <int KMAX>
 static int launch_k(const focus_shape* s, const void* h, int64_t sb, int64_t sn, int d, const float* folded, const float* bias,
                     uint32_t* mq, uint32_t* mk, unsigned long long* near_ties, float eps, float* scores, cudaStream_t st) {
-    const size_t smem = (size_t)2 * AH_THREADS * AH_ROWB + (size_t)2 * KMAX * AH_CHUNK * sizeof(float);
+    using Cfg = HiddenCfg<KMAX>;
     auto kern = assign_hidden_kernel<KMAX>;
-    int rc = check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
+    int rc = check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM_BYTES),
                         "cudaFuncSetAttribute(assign_hidden)");
     if (rc) return rc;
-    kern<<<dim3(cdiv(s->n, AH_THREADS), s->batch), AH_THREADS, smem, st>>>(
-        reinterpret_cast<const __nv_bfloat16*>(h), sb, sn, s->n, d, s->K, s->topk, folded, bias, s->Hq, s->Hkv, mq, mk, near_ties, eps,
-        scores);
+    if ((rc = check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100),
+                         "cudaFuncSetAttribute(assign_hidden)"))) return rc;
+    // one resident wave: as many blocks as fit on the device at once (fewer when there are fewer tiles).  Blocks of
+    // 128 threads per SM: by shared memory (227 KB, 1 KB reserved per block), by the 512 columns of tensor memory, at most 3
+    int dev = 0, sms = 0;
+    if ((rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice"))) return rc;
+    if ((rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "cudaDeviceGetAttribute"))) return rc;
+    int per_sm = (int)(227 * 1024 / (Cfg::SMEM_BYTES + 1024));
+    if (per_sm > (int)(512 / Cfg::TMEM_COLS)) per_sm = (int)(512 / Cfg::TMEM_COLS);
+    if (per_sm > 3) per_sm = 3;
+    if (per_sm < 1) per_sm = 1;
+    const long long resident = (long long)sms * per_sm;
+    const int ntile = cdiv(s->n, 128);
+    const long long nitems = (long long)s->batch * ntile;
+    if (nitems == 0) return 0;
+    if (nitems > 0x7fffffffll || (long long)(nitems / (nitems < resident ? nitems : resident) + 1) * cdiv(d, AH_CHUNK) > 0x7fffffffll)
+        return fail(FOCUS_ERR_UNSUPPORTED, "focus_assign_hidden: too many chunks of 128 x 128 elements for one launch");
+    const int nblocks = (int)(nitems < resident ? nitems : resident);
+    const int share = (int)(nitems / nblocks), extra = (int)(nitems % nblocks);
+    kern<<<nblocks, AH_THREADS, Cfg::SMEM_BYTES, st>>>(reinterpret_cast<const __nv_bfloat16*>(h), sb, sn, s->n, d, s->K, s->topk, folded,
+                                                       bias, s->Hq, s->Hkv, mq, mk, near_ties, eps, scores, ntile, share, extra);
     return check_cuda(cudaGetLastError(), "assign_hidden kernel launch");
 }
 
