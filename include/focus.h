@@ -187,7 +187,9 @@ FOCUS_API int focus_assign(const focus_shape* shape, focus_tensor x, int32_t H, 
  *               vectors the hidden states are scored against (each hidden state is then read once)
  *   mq_out      device uint32 [batch*Hq, n] or NULL     mk_out   device uint32 [batch*Hkv, n] or NULL
  *   near_ties   device, nullable: incremented by the number of tokens whose margin score(topk-th) - score((topk+1)-th),
- *               in fp32 and in score units, is below near_tie_eps
+ *               in fp32 and in score units, is below near_tie_eps; bit 63 is the kernel's fault flag as in focus_assign
+ * Arithmetic: as in focus_assign, the dot products run on the tensor cores with each fp32 folded value split into
+ * three bf16 terms (exact products, fp32 sums over d_model).
  */
 FOCUS_API int focus_assign_hidden(const focus_shape* shape, const void* h, int64_t stride_b, int64_t stride_n,
                                   int32_t d_model, int32_t d_g, const float* Wg, const float* C, const float* bias,

@@ -9,7 +9,9 @@
 // Scoring runs on the tensor cores.  The tiles of 128 tokens are dealt out as one contiguous range per block,
 // one resident wave of small blocks.  A block walks its tiles in chunks of 128 elements of d: the chunk of the
 // 128 rows goes to shared memory with coalesced asynchronous 16-byte copies, laid out as the K-major,
-// 128-byte-swizzled operand of a tcgen05 MMA, two chunks in flight; the same chunk of the K folded vectors is
+// 128-byte-swizzled operand of a tcgen05 MMA, in a ring of three stages (a stage is refilled as soon as the
+// MMAs of the chunk before the current one are done, so two chunks are in flight while a third is multiplied);
+// the same chunk of the K folded vectors (loaded into registers one chunk ahead) is
 // split into three bf16 terms each (hi + mid + lo carries 24 mantissa bits, so the products with the bf16 hidden
 // states sum to the fp32 dot product) as the second operand.  One thread issues the MMAs of the chunk, which
 // accumulate S = H F'^T (128 x 3K, fp32) in tensor memory over the chunks of the tile; after the last chunk every
@@ -23,22 +25,23 @@ using namespace ptx;
 
 constexpr int AH_THREADS = 128;      // one thread per token of the tile = one lane of tensor memory
 constexpr int AH_CHUNK = 128;        // elements of d per stage: two 64-column sub-tiles
+constexpr int AH_NS = 3;             // stages of the chunk ring: one being read by the MMAs, two being filled
 
 template <int KMAX>
 struct HiddenCfg {
     static constexpr int NCOLS = (3 * KMAX + 15) / 16 * 16;             // rows of F' = columns of S
     static constexpr uint32_t SUB_BYTES = 128 * 128;                     // 128 tokens x 64 elements
-    static constexpr uint32_t A_BYTES = 2 * SUB_BYTES;
+    static constexpr uint32_t A_BYTES = (AH_CHUNK / 64) * SUB_BYTES;
     static constexpr uint32_t FSUB_BYTES = NCOLS * 128;                  // NCOLS rows x 64 elements
-    static constexpr uint32_t F_BYTES = 2 * FSUB_BYTES;
+    static constexpr uint32_t F_BYTES = (AH_CHUNK / 64) * FSUB_BYTES;
     static constexpr uint32_t STAGE_BYTES = A_BYTES + F_BYTES;
     static constexpr uint32_t TMEM_COLS = NCOLS <= 32 ? 32 : (NCOLS <= 64 ? 64 : 128);
-    static constexpr uint32_t SMEM_BYTES = 2 * STAGE_BYTES + 256;
+    static constexpr uint32_t SMEM_BYTES = AH_NS * STAGE_BYTES + 256;
     static_assert(STAGE_BYTES % 1024 == 0, "every operand starts on a swizzle atom");
 };
 
 struct HiddenCtl {
-    uint64_t mma_done[2];             // the MMAs that read stage 0 / 1 have completed
+    uint64_t mma_done[AH_NS];         // the MMAs that read the stage have completed
     uint32_t tmem_base;
     int fault;
 };
@@ -63,7 +66,7 @@ assign_hidden_kernel(const __nv_bfloat16* __restrict__ h, int64_t stride_b, int6
     using Cfg = HiddenCfg<KMAX>;
     extern __shared__ __align__(1024) unsigned char sm[];
     const uint32_t base = smem_u32(sm);
-    HiddenCtl* const ctl = reinterpret_cast<HiddenCtl*>(sm + 2 * Cfg::STAGE_BYTES);
+    HiddenCtl* const ctl = reinterpret_cast<HiddenCtl*>(sm + AH_NS * Cfg::STAGE_BYTES);
     constexpr int CPR = AH_CHUNK / 8;                          // 16-byte pieces per row of a chunk
     constexpr int RSTEP = AH_THREADS / CPR;                    // rows covered by one copy per thread (8)
 
@@ -84,13 +87,25 @@ assign_hidden_kernel(const __nv_bfloat16* __restrict__ h, int64_t stride_b, int6
     // call commits one group, empty when the chunk does not exist.  (it, ic) = tile and chunk of the next call.
     const int r0 = threadIdx.x / CPR, cc = threadIdx.x % CPR;
     int it_next = 0, ic_next = 0;
+    constexpr int FPT = KMAX * AH_CHUNK / AH_THREADS;          // folded values per thread and chunk
+    float fv[FPT];                                             // those of the chunk the next call stages, loaded one call ahead
+    auto load_folded = [&]() {
+        const int e0 = ic_next * AH_CHUNK;
+#pragma unroll
+        for (int i = 0; i < FPT; ++i) {
+            const int q = i * AH_THREADS + threadIdx.x;
+            const int g = q / AH_CHUNK, e = e0 + q % AH_CHUNK;
+            fv[i] = (g < K && e < d) ? __ldg(folded + (size_t)g * d + e) : 0.f;
+        }
+    };
+    load_folded();
     auto stage_chunk = [&](int j) {
         if (j < total) {
             const int item = item0 + it_next;
             const int b = item / ntile, tok0 = (item % ntile) * 128;
             const int e0 = ic_next * AH_CHUNK;
-            unsigned char* const st = sm + (j & 1) * Cfg::STAGE_BYTES;
-            const uint32_t dstb = base + (j & 1) * Cfg::STAGE_BYTES + (cc >> 3) * Cfg::SUB_BYTES + r0 * 128 +
+            unsigned char* const st = sm + (j % AH_NS) * Cfg::STAGE_BYTES;
+            const uint32_t dstb = base + (j % AH_NS) * Cfg::STAGE_BYTES + (cc >> 3) * Cfg::SUB_BYTES + r0 * 128 +
                                   ((((uint32_t)cc & 7u) ^ ((uint32_t)r0 & 7u)) << 4);
             if (e0 + cc * 8 < d) {
                 const __nv_bfloat16* src = h + (size_t)b * stride_b + (size_t)(tok0 + r0) * stride_n + e0 + cc * 8;
@@ -108,17 +123,18 @@ assign_hidden_kernel(const __nv_bfloat16* __restrict__ h, int64_t stride_b, int6
                     asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dstb + i * RSTEP * 128), "r"(0) : "memory");
             }
             unsigned char* const fp = st + Cfg::A_BYTES;
-            const int e = e0 + threadIdx.x;
 #pragma unroll
-            for (int g = 0; g < KMAX; ++g) {
-                const float v = (g < K && e < d) ? __ldg(folded + (size_t)g * d + e) : 0.f;
+            for (int i = 0; i < FPT; ++i) {
+                const int q = i * AH_THREADS + threadIdx.x;
+                const int g = q / AH_CHUNK, col = q % AH_CHUNK;
                 __nv_bfloat16 hi, mid, lo;
-                split3_bf16(v, hi, mid, lo);
-                *reinterpret_cast<__nv_bfloat16*>(fp + sw128_offset(g, threadIdx.x, Cfg::NCOLS)) = hi;
-                *reinterpret_cast<__nv_bfloat16*>(fp + sw128_offset(KMAX + g, threadIdx.x, Cfg::NCOLS)) = mid;
-                *reinterpret_cast<__nv_bfloat16*>(fp + sw128_offset(2 * KMAX + g, threadIdx.x, Cfg::NCOLS)) = lo;
+                split3_bf16(fv[i], hi, mid, lo);
+                *reinterpret_cast<__nv_bfloat16*>(fp + sw128_offset(g, col, Cfg::NCOLS)) = hi;
+                *reinterpret_cast<__nv_bfloat16*>(fp + sw128_offset(KMAX + g, col, Cfg::NCOLS)) = mid;
+                *reinterpret_cast<__nv_bfloat16*>(fp + sw128_offset(2 * KMAX + g, col, Cfg::NCOLS)) = lo;
             }
             if (++ic_next == nchunk) { ic_next = 0; ++it_next; }
+            if (j + 1 < total) load_folded();
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
@@ -127,23 +143,23 @@ assign_hidden_kernel(const __nv_bfloat16* __restrict__ h, int64_t stride_b, int6
     {
         constexpr int ZROWS = Cfg::NCOLS - 3 * KMAX;
         if constexpr (ZROWS > 0) {
-            for (int i = threadIdx.x; i < 2 * 2 * ZROWS * 8; i += AH_THREADS) {
-                const int stg = i / (2 * ZROWS * 8), rem = i % (2 * ZROWS * 8);
+            constexpr int NSUB = AH_CHUNK / 64;
+            for (int i = threadIdx.x; i < AH_NS * NSUB * ZROWS * 8; i += AH_THREADS) {
+                const int stg = i / (NSUB * ZROWS * 8), rem = i % (NSUB * ZROWS * 8);
                 const int sub = rem / (ZROWS * 8), q = rem % (ZROWS * 8);
                 *reinterpret_cast<uint4*>(sm + stg * Cfg::STAGE_BYTES + Cfg::A_BYTES + sub * Cfg::FSUB_BYTES + (3 * KMAX) * 128 + q * 16) =
                     make_uint4(0, 0, 0, 0);
             }
         }
     }
-    stage_chunk(0);
-    stage_chunk(1);
+#pragma unroll
+    for (int j = 0; j < AH_NS - 1; ++j) stage_chunk(j);
     if (warp == 0) {
         tmem_alloc(smem_u32(&ctl->tmem_base), Cfg::TMEM_COLS);
         tmem_relinquish();
     }
     if (threadIdx.x == 32) {
-        mbar_init(smem_u32(&ctl->mma_done[0]), 1);
-        mbar_init(smem_u32(&ctl->mma_done[1]), 1);
+        for (int i = 0; i < AH_NS; ++i) mbar_init(smem_u32(&ctl->mma_done[i]), 1);
         fence_mbar_init();
         ctl->fault = 0;
     }
@@ -152,8 +168,8 @@ assign_hidden_kernel(const __nv_bfloat16* __restrict__ h, int64_t stride_b, int6
     unsigned int near_votes = 0;
     int it = 0, ic = 0;                                        // tile and chunk of iteration j
     for (int j = 0; j < total; ++j) {
-        const int buf = j & 1;
-        asm volatile("cp.async.wait_group 1;" ::: "memory");   // this thread's copies of chunk j have landed
+        const int buf = j % AH_NS;
+        asm volatile("cp.async.wait_group %0;" ::"n"(AH_NS - 2) : "memory");   // this thread's copies of chunk j have landed
         fence_proxy_async_smem();                              // generic-proxy writes before the MMA's async-proxy reads
         tc_fence_before();
         __syncthreads();
@@ -172,13 +188,20 @@ assign_hidden_kernel(const __nv_bfloat16* __restrict__ h, int64_t stride_b, int6
             }
             __syncwarp();
         }
-        if (ok && !mbar_wait(smem_u32(&ctl->mma_done[buf]), (uint32_t)((j >> 1) & 1))) {
+        // the stage chunk j - 1 was read from is free once its MMAs are done (long ago, as a rule): refill it while
+        // the MMAs of chunk j run
+        if (ok && j > 0 && !mbar_wait(smem_u32(&ctl->mma_done[(j - 1) % AH_NS]), (uint32_t)(((j - 1) / AH_NS) & 1))) {
             ok = false;
             ctl->fault = 1;
         }
+        stage_chunk(j + AH_NS - 1);
         const bool last_chunk = ic == nchunk - 1;
         float sc3[Cfg::NCOLS];
         if (last_chunk) {
+            if (ok && !mbar_wait(smem_u32(&ctl->mma_done[buf]), (uint32_t)((j / AH_NS) & 1))) {
+                ok = false;
+                ctl->fault = 1;
+            }
             tc_fence_after();
             if (ok) {
 #pragma unroll
@@ -195,8 +218,6 @@ assign_hidden_kernel(const __nv_bfloat16* __restrict__ h, int64_t stride_b, int6
             }
             tc_fence_before();
         }
-        __syncthreads();                                       // the stage is free: its MMAs are done
-        stage_chunk(j + 2);
 
         if (last_chunk) {
             const int item = item0 + it;
