@@ -331,7 +331,8 @@ def main():
         def timed_alone(fn, reps=5):
             ts = []
             for i in range(reps + 1):
-                flush.zero_()
+                flush.zero_()                       # evicts what the last launch left in L2 ...
+                flush.view(torch.int64).sum()       # ... and reading it back leaves clean lines: no write-backs under the timed launch
                 a, b = ev(), ev()
                 a.record(); fn(); b.record()
                 torch.cuda.synchronize()
@@ -356,7 +357,7 @@ def main():
             gbs = (rows * 4 * wl.D + wl.Hkv * max(far, 0) * 4) / (ms * 1e-3) / 1e9
             extra["focus_decode_step"] = dict(bound="hbm", ms=ms, achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s",
                                               frac=gbs / peaks["hbm_gbs"], kv_rows_read=rows, kv_rows_total=wl.Hkv * wl.n,
-                                              note="bytes = 4 D per attended (KV head, key) + 4 per far key mask; L2 flushed")
+                                              note="bytes = 4 D per attended (KV head, key) + 4 per far key mask; L2 flushed (256 MiB written, then read back)")
         d_model, d_g = 4096, 16
         gen = torch.Generator(device="cuda"); gen.manual_seed(7)
         hid = torch.randn((1, wl.n, d_model), generator=gen, device="cuda").to(torch.bfloat16)
