@@ -333,9 +333,10 @@ FOCUS_API int focus_count_kept_noalloc(const focus_shape* shape, const uint32_t*
  * followed as printed: two orthogonal assignments give the gate sigmoid(0) = 1/2.  Same kernel, operand
  * precision and accumulation as focus_attn_fwd in dense causal mode; the gate is evaluated in fp32 as
  * 1/2 + 1/2 tanh(lambda/2 g_i.g_j) with the hardware tanh approximation.
- *   shape       softcap must be 0; K <= 8 (FOCUS_ERR_UNSUPPORTED otherwise); masks and topk are not used
+ *   shape       softcap must be 0; K <= 32, and K <= 16 at D = 256 (FOCUS_ERR_UNSUPPORTED otherwise); masks and topk
+ *               are not used
  *   q, k, v, o, lse, dev_status   as for focus_attn_fwd
- *   g           device fp32 [batch, n, ld], ld = 4 (K <= 4) or 8; one assignment per token, shared by all heads;
+ *   g           device fp32 [batch, n, ld], ld = focus_soft_ld(K) (4, 8, 16 or 32); one assignment per token, shared by all heads;
  *               entries g >= K must be 0 (focus_sinkhorn writes them so); 16-byte aligned
  */
 FOCUS_API int focus_router_scores(const focus_shape* shape, const void* h, int64_t stride_b, int64_t stride_n,

@@ -384,7 +384,8 @@ int focus_gate_attn_fwd(const focus_shape* shape, focus_tensor q, focus_tensor k
     if (!lse || !g) return fail(FOCUS_ERR_INVALID_ARG, "lse or g is NULL");
     if ((uintptr_t)g % 16) return fail(FOCUS_ERR_INVALID_ARG, "g is not 16-byte aligned");
     if (shape->softcap > 0.f) return fail(FOCUS_ERR_UNSUPPORTED, "the gated forward takes no softcap");
-    if (shape->K > 8) return fail(FOCUS_ERR_UNSUPPORTED, "the gated forward supports K <= 8 (K = %d)", shape->K);
+    if (shape->K > 32 || (shape->D == 256 && shape->K > 16))
+        return fail(FOCUS_ERR_UNSUPPORTED, "the gated forward supports K <= 32 (K <= 16 at D = 256); K = %d", shape->K);
     if ((rc = require_sm100())) return rc;
     AttnArgs a;
     a.s = *shape;

@@ -33,7 +33,8 @@
 
 namespace focus {
 
-template <int D, bool GATE = false>
+// GATE: 0 = no soft gate, else the number of 8-float chunks of a token's soft assignment (1, 2 or 4: K <= 8, 16, 32)
+template <int D, int GATE = 0>
 struct AttnCfg {
     static constexpr int NQ = (D == 256) ? 1 : 2;            // 128-row query tiles per item
     static constexpr int SUBT = D / 64;
@@ -45,9 +46,11 @@ struct AttnCfg {
     // all 256 dimensions.  Five half stages fit, and a half goes back to the producer as soon as its own MMAs are done.
     static constexpr int PARTS = (D == 256) ? 2 : 1;         // ring stages per tile
     static constexpr uint32_t STAGE_BYTES = TILE_BYTES / PARTS;
-    static constexpr int NSTAGE = (D == 256) ? (GATE ? 4 : 5) : ((D == 128) ? (GATE ? 4 : 5) : 8);
-    // soft gate: per softmax warpgroup two buffers of 128 key assignments, 8 floats each (after the ring)
-    static constexpr uint32_t GATE_BUF_BYTES = 128 * 32;
+    static constexpr int NSTAGE = (D == 256) ? (GATE ? 4 : 5) : ((D == 128) ? (GATE == 4 ? 3 : (GATE ? 4 : 5)) : 8);
+    // soft gate: per softmax warpgroup two buffers of 128 key assignments, 8 GATE floats each (after the ring)
+    static constexpr uint32_t GATE_ROW_BYTES = 32 * (GATE ? GATE : 1);
+    static constexpr uint32_t GATE_BUF_BYTES = 128 * GATE_ROW_BYTES;
+    static_assert(!(D == 256 && GATE == 4), "no room for the K/V ring beside 64 KB of gate buffers at D = 256");
     static constexpr uint32_t SMEM_BYTES = 1024 + NQ * TILE_BYTES + NSTAGE * STAGE_BYTES + (GATE ? 4 * GATE_BUF_BYTES : 0);
     // Ring order of the tiles.  With one query tile the S of the next key tile is issued before the current P V, so
     // K(next) travels ahead of V(current); with two query tiles V(current) is consumed and released first.
@@ -95,7 +98,7 @@ __device__ __forceinline__ void report_timeout(const AttnParams& p, SharedCtl* c
     }
 }
 
-template <int D, bool SOFTCAP, bool GATE>
+template <int D, bool SOFTCAP, int GATE>
 __global__ void __launch_bounds__(AttnCfg<D, GATE>::THREADS, 1)
 focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
@@ -433,15 +436,20 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             float m_used = -INFINITY, l = 0.f;
             bool first = true;
             // soft gate: this row's assignment times lambda / 2 (sigmoid(x) = 1/2 + 1/2 tanh(x / 2))
-            float gi[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            if constexpr (GATE) {
+            constexpr int GQ = GATE ? 2 * GATE : 2;               // 16-byte pieces of an assignment row held per token
+            float gi[4 * GQ];
+#pragma unroll
+            for (int e = 0; e < 4 * GQ; ++e) gi[e] = 0.f;
+            if constexpr (GATE != 0) {
                 if (valid) {
                     const float4* gp = reinterpret_cast<const float4*>(p.gate_g + ((size_t)bb * p.n + (size_t)i) * p.gate_ld);
-                    const float4 g0 = __ldg(gp);
-                    gi[0] = g0.x * p.gate_hl; gi[1] = g0.y * p.gate_hl; gi[2] = g0.z * p.gate_hl; gi[3] = g0.w * p.gate_hl;
-                    if (p.gate_ld == 8) {
-                        const float4 g1 = __ldg(gp + 1);
-                        gi[4] = g1.x * p.gate_hl; gi[5] = g1.y * p.gate_hl; gi[6] = g1.z * p.gate_hl; gi[7] = g1.w * p.gate_hl;
+#pragma unroll
+                    for (int f = 0; f < GQ; ++f) {
+                        if (4 * f < p.gate_ld) {
+                            const float4 g0 = __ldg(gp + f);
+                            gi[4 * f] = g0.x * p.gate_hl; gi[4 * f + 1] = g0.y * p.gate_hl;
+                            gi[4 * f + 2] = g0.z * p.gate_hl; gi[4 * f + 3] = g0.w * p.gate_hl;
+                        }
                     }
                 }
             }
@@ -463,7 +471,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 bool gated = false;
                 const long long gj0 = (long long)kb * 128 + half * NC;    // first column of this thread's part of the tile
                 const long long ifar = i - p.w;                           // columns j < ifar are distant for this row
-                if constexpr (GATE) {
+                if constexpr (GATE != 0) {
                     // the same decision in all four warps of the warpgroup: does the tile hold a distant pair at all
                     const bool tile_gated = !tm.all_masked && ((long long)a * 128 + 127 - p.w > gj0);
                     if (tile_gated) {
@@ -472,8 +480,9 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         if (col < NC) {
                             const long long j = gj0 + col;
                             const float4* gp = reinterpret_cast<const float4*>(p.gate_g + ((size_t)bb * p.n + (size_t)(j < p.n ? j : p.n - 1)) * p.gate_ld);
-                            reinterpret_cast<float4*>(gw + col * 32)[0] = __ldg(gp);
-                            reinterpret_cast<float4*>(gw + col * 32)[1] = p.gate_ld == 8 ? __ldg(gp + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                            for (int f = 0; f < GQ; ++f)
+                                reinterpret_cast<float4*>(gw + col * C::GATE_ROW_BYTES)[f] = 4 * f < p.gate_ld ? __ldg(gp + f) : make_float4(0.f, 0.f, 0.f, 0.f);
                         }
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&ctl.gbar[wg]));
@@ -499,31 +508,52 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
                     for (int c = 0; c < NC / 32; ++c) {
                         tmem_ld32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[c * 32]));
-                        if constexpr (GATE) {       // chunk by chunk: 32 scores, then their factors
+                        if constexpr (GATE != 0) {       // chunk by chunk: 32 scores, then their factors
                             tmem_wait_ld();
                             if (gated) {
                                 const bool wide = p.gate_ld == 8;
                                 const int nfar = (int)(ifar - gj0 < 0 ? 0 : (ifar - gj0 > NC ? NC : ifar - gj0));   // columns < nfar are distant
 #pragma unroll
                                 for (int e0 = 0; e0 < 32; e0 += 4) {        // four columns in flight
-                                    float4 k0[4], k1[4];
-#pragma unroll
-                                    for (int u = 0; u < 4; ++u) {
-                                        const float4* kp = reinterpret_cast<const float4*>(gb + (c * 32 + e0 + u) * 32);
-                                        k0[u] = kp[0];
-                                        k1[u] = wide ? kp[1] : make_float4(0.f, 0.f, 0.f, 0.f);
-                                    }
                                     float arg[4];
+                                    if constexpr (GATE == 1) {
+                                        float4 k0[4], k1[4];
 #pragma unroll
-                                    for (int u = 0; u < 4; ++u) {
-                                        float2 acc = __fmul2_rn(make_float2(gi[0], gi[1]), make_float2(k0[u].x, k0[u].y));
-                                        acc = __ffma2_rn(make_float2(gi[2], gi[3]), make_float2(k0[u].z, k0[u].w), acc);
-                                        if (wide) {
-                                            float2 acb = __fmul2_rn(make_float2(gi[4], gi[5]), make_float2(k1[u].x, k1[u].y));
-                                            acb = __ffma2_rn(make_float2(gi[6], gi[7]), make_float2(k1[u].z, k1[u].w), acb);
-                                            acc = __fadd2_rn(acc, acb);
+                                        for (int u = 0; u < 4; ++u) {
+                                            const float4* kp = reinterpret_cast<const float4*>(gb + (c * 32 + e0 + u) * 32);
+                                            k0[u] = kp[0];
+                                            k1[u] = wide ? kp[1] : make_float4(0.f, 0.f, 0.f, 0.f);
                                         }
-                                        arg[u] = acc.x + acc.y;
+#pragma unroll
+                                        for (int u = 0; u < 4; ++u) {
+                                            float2 acc = __fmul2_rn(make_float2(gi[0], gi[1]), make_float2(k0[u].x, k0[u].y));
+                                            acc = __ffma2_rn(make_float2(gi[2], gi[3]), make_float2(k0[u].z, k0[u].w), acc);
+                                            if (wide) {
+                                                float2 acb = __fmul2_rn(make_float2(gi[4], gi[5]), make_float2(k1[u].x, k1[u].y));
+                                                acb = __ffma2_rn(make_float2(gi[6], gi[7]), make_float2(k1[u].z, k1[u].w), acb);
+                                                acc = __fadd2_rn(acc, acb);
+                                            }
+                                            arg[u] = acc.x + acc.y;
+                                        }
+                                    } else {
+                                        // longer assignments: piece by piece, two sums per column
+                                        float2 acc[4], acb[4];
+#pragma unroll
+                                        for (int u = 0; u < 4; ++u) acc[u] = acb[u] = make_float2(0.f, 0.f);
+#pragma unroll
+                                        for (int f = 0; f < GQ; ++f) {
+                                            float4 kf[4];
+#pragma unroll
+                                            for (int u = 0; u < 4; ++u)
+                                                kf[u] = reinterpret_cast<const float4*>(gb + (c * 32 + e0 + u) * C::GATE_ROW_BYTES)[f];
+#pragma unroll
+                                            for (int u = 0; u < 4; ++u) {
+                                                acc[u] = __ffma2_rn(make_float2(gi[4 * f], gi[4 * f + 1]), make_float2(kf[u].x, kf[u].y), acc[u]);
+                                                acb[u] = __ffma2_rn(make_float2(gi[4 * f + 2], gi[4 * f + 3]), make_float2(kf[u].z, kf[u].w), acb[u]);
+                                            }
+                                        }
+#pragma unroll
+                                        for (int u = 0; u < 4; ++u) arg[u] = (acc[u].x + acc[u].y) + (acb[u].x + acb[u].y);
                                     }
 #pragma unroll
                                     for (int u = 0; u < 4; ++u) {
@@ -694,7 +724,7 @@ focus_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
-template <int D, bool SOFTCAP, bool GATE>
+template <int D, bool SOFTCAP, int GATE>
 static int launch_attn_t(const AttnArgs& a, cudaStream_t st) {
     using C = AttnCfg<D, GATE>;
     CUtensorMap tq, tk, tv;
@@ -790,16 +820,19 @@ int launch_attn_sm100(const AttnArgs& a, cudaStream_t st) {
 static int launch_attn_one(const AttnArgs& a, cudaStream_t st) {
     const bool cap = a.s.softcap > 0.f;
     if (a.gate_g) {      // training-time gated forward: dense causal walk, no softcap
+        const int chunks = a.gate_ld <= 8 ? 1 : a.gate_ld / 8;      // 8-float chunks of an assignment row
         switch (a.s.D) {
-            case 64: return launch_attn_t<64, false, true>(a, st);
-            case 128: return launch_attn_t<128, false, true>(a, st);
-            case 256: return launch_attn_t<256, false, true>(a, st);
+            case 64: return chunks == 1 ? launch_attn_t<64, false, 1>(a, st) : chunks == 2 ? launch_attn_t<64, false, 2>(a, st) : launch_attn_t<64, false, 4>(a, st);
+            case 128: return chunks == 1 ? launch_attn_t<128, false, 1>(a, st) : chunks == 2 ? launch_attn_t<128, false, 2>(a, st) : launch_attn_t<128, false, 4>(a, st);
+            case 256:
+                if (chunks == 4) return fail(FOCUS_ERR_UNSUPPORTED, "the gated forward at D = 256 supports K <= 16");
+                return chunks == 1 ? launch_attn_t<256, false, 1>(a, st) : launch_attn_t<256, false, 2>(a, st);
         }
     }
     switch (a.s.D) {
-        case 64: return cap ? launch_attn_t<64, true, false>(a, st) : launch_attn_t<64, false, false>(a, st);
-        case 128: return cap ? launch_attn_t<128, true, false>(a, st) : launch_attn_t<128, false, false>(a, st);
-        case 256: return cap ? launch_attn_t<256, true, false>(a, st) : launch_attn_t<256, false, false>(a, st);
+        case 64: return cap ? launch_attn_t<64, true, 0>(a, st) : launch_attn_t<64, false, 0>(a, st);
+        case 128: return cap ? launch_attn_t<128, true, 0>(a, st) : launch_attn_t<128, false, 0>(a, st);
+        case 256: return cap ? launch_attn_t<256, true, 0>(a, st) : launch_attn_t<256, false, 0>(a, st);
     }
     return fail(FOCUS_ERR_UNSUPPORTED, "D (%d) must be 64, 128 or 256", a.s.D);
 }

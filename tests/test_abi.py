@@ -145,8 +145,9 @@ def test_training_forward_host_checks():
     assert L.focus_gate_attn_fwd(ctypes.byref(s), t_ok, t_ok, t_ok, 4100, 5.0, t_ok, 4096, None, None) == -1     # g alignment
     capped = fb.make_shape(8, 2, 1000, 128, 8, 2, 64, softcap=30.0)
     assert L.focus_gate_attn_fwd(ctypes.byref(capped), t_ok, t_ok, t_ok, 4096, 5.0, t_ok, 4096, None, None) == -2   # unsupported
-    many = fb.make_shape(8, 2, 1000, 128, 16, 2, 64)
-    assert L.focus_gate_attn_fwd(ctypes.byref(many), t_ok, t_ok, t_ok, 4096, 5.0, t_ok, 4096, None, None) == -2
+    many = fb.make_shape(8, 2, 1000, 256, 32, 2, 64)       # D = 256 leaves no room for 32-float assignment rows
+    t256 = fb.focus_tensor(4096, 8 * 1000 * 256, 1000 * 256, 256)
+    assert L.focus_gate_attn_fwd(ctypes.byref(many), t256, t256, t256, 4096, 5.0, t256, 4096, None, None) == -2
 
 
 def test_tensor_arguments_that_would_alias_or_misalign_are_refused():

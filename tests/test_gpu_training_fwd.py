@@ -105,7 +105,12 @@ def check_gate(Q, Kt, V, gt, K, w, lam, O, lse, rows=None):
 @pytest.mark.parametrize("Hq,Hkv,n,D,K,w,lam,batch", [(2, 2, 1, 64, 4, 0, 5.0, 1), (4, 2, 700, 64, 4, 64, 8.0, 1), (4, 2, 1000, 128, 4, 0, 5.0, 1),
                                                       (4, 1, 1500, 128, 8, 300, 20.0, 1), (2, 1, 900, 256, 8, 100, 10.0, 1),
                                                       (2, 2, 640, 128, 5, 2000, 10.0, 1), (2, 1, 517, 128, 2, 33, 6.0, 2),
-                                                      (2, 2, 384, 256, 4, 0, 30.0, 2)])
+                                                      (2, 2, 384, 256, 4, 0, 30.0, 2),
+                                                      # assignment rows of 16 and 32 floats (K up to 32, the paper's widest ablation)
+                                                      (2, 1, 700, 128, 12, 64, 10.0, 1), (2, 2, 900, 128, 16, 0, 8.0, 1),
+                                                      (4, 2, 1100, 128, 32, 200, 10.0, 1), (2, 1, 520, 64, 32, 50, 12.0, 2),
+                                                      (2, 1, 600, 64, 9, 0, 5.0, 1), (2, 1, 777, 256, 16, 100, 10.0, 1),
+                                                      (2, 2, 300, 256, 11, 0, 20.0, 1), (2, 1, 1, 128, 32, 0, 5.0, 1)])
 def test_gated_attention_all_rows(Hq, Hkv, n, D, K, w, lam, batch):
     Q, Kt, V, gt = gate_case(Hq, Hkv, n, D, K, 100 + n, batch)
     O, lse = run_gate(Q, Kt, V, gt, K, w, lam)
@@ -118,6 +123,26 @@ def test_gate_changes_the_result():
     O, _ = run_gate(Q, Kt, V, gt, 4, 16, 10.0)
     O2, _ = run_gate(Q, Kt, V, gt, 4, 5000, 10.0)
     assert (O.float() - O2.float()).abs().max().item() > 0.2
+
+
+def test_gated_attention_refuses_what_it_has_no_room_for():
+    """D = 256 with more than 16 groups: the gate buffers would leave no room for the K/V ring"""
+    Q, Kt, V, gt = gate_case(2, 1, 256, 256, 32, 9)
+    shape = fb.make_shape(2, 1, 256, 256, 32, 1, 16)
+    O = torch.empty_like(Q); lse = torch.empty((2, 256), dtype=torch.float32, device="cuda")
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    with pytest.raises(fb.FocusError, match="K <= 16 at D = 256"):
+        fb.focus_gate_attn_fwd(shape, Q, Kt, V, gt, 5.0, O, lse, status)
+
+
+def test_gated_attention_32_groups_sampled_rows():
+    """K = 32 at a length with several items per CTA (three-stage K/V ring beside the gate buffers)"""
+    n, K, w, lam = 20000, 32, 1024, 10.0
+    Q, Kt, V, gt = gate_case(4, 2, n, 128, K, 57)
+    O, lse = run_gate(Q, Kt, V, gt, K, w, lam)
+    rng = np.random.default_rng(6)
+    rows = np.unique(np.concatenate([rng.integers(0, n, 12), [0, w, w + 1, n - 1]]))
+    check_gate(Q, Kt, V, gt, K, w, lam, O, lse, rows)
 
 
 @pytest.mark.parametrize("D,n", [(128, 40000), (256, 20000)])
@@ -136,8 +161,6 @@ def test_refusals():
     O = torch.empty_like(Q); lse = torch.empty((2, 256), dtype=torch.float32, device="cuda")
     with pytest.raises(fb.FocusError):      # softcap
         fb.focus_gate_attn_fwd(fb.make_shape(2, 2, 256, 128, 4, 1, 16, softcap=30.0), Q, Kt, V, gt, 5.0, O, lse)
-    with pytest.raises(fb.FocusError):      # more groups than the gated forward takes
-        fb.focus_gate_attn_fwd(fb.make_shape(2, 2, 256, 128, 16, 1, 16), Q, Kt, V, gt, 5.0, O, lse)
     shape = fb.make_shape(2, 2, 256, 128, 4, 1, 16)
     small = torch.empty(8, dtype=torch.uint8, device="cuda")
     with pytest.raises(fb.FocusError):      # workspace too small
