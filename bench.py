@@ -376,10 +376,17 @@ def main():
         soft = torch.empty((1, wl.n, ld), dtype=torch.float32, device="cuda")
         ws_sk = torch.empty(fb.focus_sinkhorn_workspace_bytes(shape, 10), dtype=torch.uint8, device="cuda")
         ms_sc = timed_alone(lambda: fb.focus_router_scores(shape, hid, Wg, Cg, folded, soft))
+        scores = soft.clone()
         ms_sk = timed_alone(lambda: fb.focus_sinkhorn(shape, soft, 0.1, 10, ws_sk, soft))
-        tr = dict(router_scores_ms=ms_sc, sinkhorn_ms=ms_sk,
-                  note="tau = 0.1, 10 Sinkhorn iterations (12 small launches on an L2-resident score matrix), lambda = 10")
-        if wl.K <= 8 and wl.softcap == 0:
+        ws_skb = torch.empty(fb.focus_sinkhorn_bwd_workspace_bytes(shape, 10), dtype=torch.uint8, device="cuda")
+        dsoft = torch.randn(soft.shape, generator=gen, device="cuda")
+        dscores = torch.empty_like(soft)
+        ms_skb = timed_alone(lambda: fb.focus_sinkhorn_bwd(shape, scores, 0.1, 10, ws_skb, dsoft, dscores))
+        del scores, dsoft, dscores
+        tr = dict(router_scores_ms=ms_sc, sinkhorn_ms=ms_sk, sinkhorn_bwd_ms=ms_skb,
+                  note="tau = 0.1, 10 Sinkhorn iterations (12 small launches on an L2-resident score matrix; the backward "
+                       "repeats the column sums and adds 11 launches), lambda = 10")
+        if wl.softcap == 0 and (wl.K <= 16 or wl.D < 256):
             O_g, lse_g = torch.empty_like(Q), torch.empty_like(lse)
             ms_g = timed_alone(lambda: fb.focus_gate_attn_fwd(shape, Q, K, V, soft, 10.0, O_g, lse_g, status), reps=2)
             del O_g, lse_g

@@ -351,6 +351,24 @@ FOCUS_API int focus_gate_attn_fwd(const focus_shape* shape, focus_tensor q, focu
                                   void* stream);
 
 /*
+ * focus_sinkhorn_bwd -- the derivative of focus_sinkhorn (paper Sec. 2 "Learned grouping": the soft assignments are
+ * trained through the Sinkhorn steps).  Given dg = d loss / d g for g = sinkhorn(scores, tau, iters), writes
+ * d loss / d scores.  Each step "divide by the sum along an axis", Z = X / sum(X), is differentiated as
+ * dX = (dZ - sum(dZ * Z)) / sum(X) along that axis, the `iters` column and row divisions in reverse order, and the
+ * exponential last: dS = dQ0 * exp(S / tau) / tau.  The iterates are not stored: a row of any iterate follows from its
+ * score row and the column sums of the forward passes, which this call recomputes into `ws` first (it does not need
+ * focus_sinkhorn to have run).  fp32 per row, column sums in fp64; offsets kept as logarithms as in the forward.
+ *   scores       device fp32 [batch, n, ld], ld = focus_soft_ld(K), as given to focus_sinkhorn; read only
+ *   ws           device scratch, focus_sinkhorn_bwd_workspace_bytes(shape, iters) bytes, 16-byte aligned
+ *   dg           device fp32 [batch, n, ld]; entries g >= K are ignored
+ *   dscores_out  device fp32 [batch, n, ld]; entries g >= K are written as 0; may be the dg buffer, not the scores
+ * The derivatives of the gated attention itself (Eq. 2) have an oracle and pins only; no kernel computes them.
+ */
+FOCUS_API size_t focus_sinkhorn_bwd_workspace_bytes(const focus_shape* shape, int32_t iters);
+FOCUS_API int focus_sinkhorn_bwd(const focus_shape* shape, const float* scores, float tau, int32_t iters, void* ws,
+                                 size_t ws_bytes, const float* dg, float* dscores_out, void* stream);
+
+/*
  * focus_selftest_umma -- diagnostic, not on the hot path (the paper has no counterpart): one
  * 128 x 128 x D tile S = A B^T and one 128 x D x 128 tile O = P V through the same TMA, descriptor
  * and tcgen05 building blocks as focus_attn_fwd, so that an encoding mistake shows up in isolation.

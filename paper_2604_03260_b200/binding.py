@@ -92,6 +92,10 @@ def lib():
         L.focus_sinkhorn_workspace_bytes.argtypes = [SP, i32]
         L.focus_sinkhorn.restype = C.c_int
         L.focus_sinkhorn.argtypes = [SP, vp, f32, i32, vp, sz, vp, vp]
+        L.focus_sinkhorn_bwd_workspace_bytes.restype = sz
+        L.focus_sinkhorn_bwd_workspace_bytes.argtypes = [SP, i32]
+        L.focus_sinkhorn_bwd.restype = C.c_int
+        L.focus_sinkhorn_bwd.argtypes = [SP, vp, f32, i32, vp, sz, vp, vp, vp]
         L.focus_gate_attn_fwd.restype = C.c_int
         L.focus_gate_attn_fwd.argtypes = [SP, focus_tensor, focus_tensor, focus_tensor, vp, f32, focus_tensor, vp, vp, vp]
         L.focus_count_kept.restype = C.c_int
@@ -213,6 +217,16 @@ def focus_sinkhorn(shape, scores, tau, iters, ws, g_out, stream=None):
     """scores, g_out fp32 [batch, n, focus_soft_ld(K)] (may be the same tensor); ws uint8 scratch"""
     _check(lib().focus_sinkhorn(C.byref(shape), _p(scores), tau, iters, _p(ws), ws.numel() * ws.element_size(), _p(g_out),
                                 _stream(stream)))
+
+
+def focus_sinkhorn_bwd_workspace_bytes(shape, iters) -> int:
+    return int(lib().focus_sinkhorn_bwd_workspace_bytes(C.byref(shape), iters))
+
+
+def focus_sinkhorn_bwd(shape, scores, tau, iters, ws, dg, dscores_out, stream=None):
+    """scores, dg, dscores_out fp32 [batch, n, focus_soft_ld(K)] (dscores_out may be dg); ws uint8 scratch"""
+    _check(lib().focus_sinkhorn_bwd(C.byref(shape), _p(scores), tau, iters, _p(ws), ws.numel() * ws.element_size(), _p(dg),
+                                    _p(dscores_out), _stream(stream)))
 
 
 def focus_gate_attn_fwd(shape, q, k, v, g, lam, o, lse, dev_status=None, stream=None):

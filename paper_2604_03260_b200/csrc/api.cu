@@ -258,6 +258,27 @@ int focus_sinkhorn(const focus_shape* shape, const float* scores, float tau, int
     return launch_sinkhorn(shape, scores, tau, iters, ws, g_out, (cudaStream_t)stream);
 }
 
+size_t focus_sinkhorn_bwd_workspace_bytes(const focus_shape* shape, int32_t iters) {
+    if (validate_shape(shape) || iters < 1) return 0;
+    return sinkhorn_bwd_workspace_bytes(shape, iters);
+}
+
+int focus_sinkhorn_bwd(const focus_shape* shape, const float* scores, float tau, int32_t iters, void* ws, size_t ws_bytes,
+                       const float* dg, float* dscores_out, void* stream) {
+    int rc = validate_shape(shape);
+    if (rc) return rc;
+    if (!scores || !ws || !dg || !dscores_out) return fail(FOCUS_ERR_INVALID_ARG, "scores, ws, dg or dscores_out is NULL");
+    if (!(tau > 0.f) || iters < 1 || iters > 1000) return fail(FOCUS_ERR_INVALID_ARG, "tau must be positive and iters in [1, 1000]");
+    if ((uintptr_t)scores % 16 || (uintptr_t)dg % 16 || (uintptr_t)dscores_out % 16 || (uintptr_t)ws % 16)
+        return fail(FOCUS_ERR_INVALID_ARG, "scores, dg, dscores_out and ws must be 16-byte aligned");
+    if (dscores_out == scores) return fail(FOCUS_ERR_INVALID_ARG, "dscores_out must not be the scores buffer (the scores are read by every pass)");
+    if (ws_bytes < sinkhorn_bwd_workspace_bytes(shape, iters))
+        return fail(FOCUS_ERR_CAPACITY, "sinkhorn backward workspace has %zu bytes, %zu needed", ws_bytes,
+                    sinkhorn_bwd_workspace_bytes(shape, iters));
+    if ((rc = require_sm100())) return rc;
+    return launch_sinkhorn_bwd(shape, scores, tau, iters, ws, dg, dscores_out, (cudaStream_t)stream);
+}
+
 int focus_build_tiles(const focus_shape* shape, const uint32_t* mq, const uint32_t* mk, int32_t layout, void* ws,
                       size_t ws_bytes, void* stream) {
     focus_tiles_layout L;

@@ -57,6 +57,9 @@ int launch_assign_hidden(const focus_shape* s, const void* h, int64_t sb, int64_
                          unsigned long long* near_ties, float eps, float* scores, cudaStream_t st);
 size_t sinkhorn_workspace_bytes(const focus_shape* s, int iters);
 int launch_sinkhorn(const focus_shape* s, const float* S, float tau, int iters, void* ws, float* out, cudaStream_t st);
+size_t sinkhorn_bwd_workspace_bytes(const focus_shape* s, int iters);
+int launch_sinkhorn_bwd(const focus_shape* s, const float* S, float tau, int iters, void* ws, const float* dG, float* dS,
+                        cudaStream_t st);
 size_t decode_workspace_bytes(const focus_shape* s);
 int launch_decode(const focus_shape* s, const focus_tensor& q, const focus_tensor& k, const focus_tensor& v,
                   const uint32_t* mq_new, const uint32_t* mk, const focus_tensor& o, float* lse, float* part, float scale,

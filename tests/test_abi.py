@@ -132,6 +132,11 @@ def test_training_forward_host_checks():
     w10, w20 = fb.focus_sinkhorn_workspace_bytes(s, 10), fb.focus_sinkhorn_workspace_bytes(s, 20)
     assert w10 > 0 and w20 > w10 and w10 % 16 == 0
     assert fb.focus_sinkhorn_workspace_bytes(s, 0) == 0
+    wb = fb.focus_sinkhorn_bwd_workspace_bytes(s, 10)
+    assert wb == w10 + 3 * 10 * 32 * 8 and fb.focus_sinkhorn_bwd_workspace_bytes(s, 0) == 0
+    assert L.focus_sinkhorn_bwd(ctypes.byref(s), 4096, 0.1, 10, 4096, wb, None, 8192, None) == -1       # dg NULL
+    assert L.focus_sinkhorn_bwd(ctypes.byref(s), 4096, 0.1, 10, 4096, wb, 8192, 4096, None) == -1       # output over the scores
+    assert L.focus_sinkhorn_bwd(ctypes.byref(s), 4096, 0.1, 10, 4096, w10, 8192, 8192, None) == -3      # capacity
     assert fb.focus_sinkhorn_workspace_bytes(fb.make_shape(8, 2, 1000, 128, 8, 2, 64, batch=1), 10) * 3 == w10   # per sequence
     assert L.focus_sinkhorn(ctypes.byref(s), None, 0.1, 10, 4096, w10, 4096, None) == -1          # scores NULL
     assert L.focus_sinkhorn(ctypes.byref(s), 4096, 0.0, 10, 4096, w10, 4096, None) == -1           # temperature

@@ -203,6 +203,53 @@ def test_gated_attention_at_the_metric_point_shape():
     check_gate(Q, Kt, V, gt, K, w, lam, O, lse, rows)
 
 
+@pytest.mark.parametrize("n,K,tau,iters,batch,spread", [(1, 4, 0.1, 10, 1, 0.3), (300, 4, 0.5, 10, 1, 1.0), (5000, 8, 0.1, 10, 1, 0.3),
+                                                        (70000, 8, 0.1, 10, 1, 0.3), (777, 32, 0.1, 3, 2, 0.5), (513, 1, 0.1, 2, 1, 1.0),
+                                                        (1000, 5, 0.1, 1, 3, 0.3), (4096, 8, 0.1, 10, 1, 10.0), (2000, 12, 0.2, 6, 1, 0.5)])
+def test_sinkhorn_backward(n, K, tau, iters, batch, spread):
+    """d loss / d scores through the Sinkhorn steps against the oracle's tape-based derivative (fp64); the oracle's
+    derivative is pinned on the CPU by central differences of its own forward"""
+    g = torch.Generator(device="cuda"); g.manual_seed(n * 11 + K)
+    ld = fb.focus_soft_ld(K)
+    S = padded(spread * torch.randn((batch, n, K), generator=g, device="cuda"), ld)
+    dG = padded(torch.randn((batch, n, K), generator=g, device="cuda"), ld)
+    dG[..., K:] = 7.0                                    # entries beyond K are ignored
+    shape = fb.make_shape(4, 2, n, 128, K, 1, 16, batch=batch)
+    ws = torch.empty(fb.focus_sinkhorn_bwd_workspace_bytes(shape, iters), dtype=torch.uint8, device="cuda")
+    dS = torch.full_like(S, float("nan"))
+    fb.focus_sinkhorn_bwd(shape, S, tau, iters, ws, dG, dS)
+    torch.cuda.synchronize()
+    got = dS.cpu().numpy().astype(np.float64)
+    assert (got[..., K:] == 0).all()
+    Sh, dGh = S.cpu().numpy().astype(np.float64), dG.cpu().numpy().astype(np.float64)
+    for b in range(batch):
+        ref = fo.sinkhorn_backward(Sh[b, :, :K], tau, iters, dGh[b, :, :K])
+        scale = max(np.abs(ref).max(), 1e-30)
+        err = np.abs(got[b, :, :K] - ref).max() / scale
+        # fp32 rows (exp, a K-term dot product with cancellation) against fp64; column sums are fp64 on both sides
+        assert err <= 2e-4, (err, scale)
+    # in place over dg, and twice in a row into the same workspace
+    fb.focus_sinkhorn_bwd(shape, S, tau, iters, ws, dG, dG)
+    torch.cuda.synchronize()
+    assert torch.equal(dG, dS)
+
+
+def test_sinkhorn_backward_is_orthogonal_to_what_sinkhorn_ignores():
+    """adding a constant to a column of the scores scales that column of exp(S / tau), which the first column division
+    undoes: the assignments do not change, so the derivative sums to zero over every column"""
+    n, K, tau, iters = 3000, 8, 0.1, 10
+    g = torch.Generator(device="cuda"); g.manual_seed(3)
+    S = 0.5 * torch.randn((1, n, 8), generator=g, device="cuda")
+    dG = torch.randn((1, n, 8), generator=g, device="cuda")
+    shape = fb.make_shape(4, 2, n, 128, K, 1, 16)
+    ws = torch.empty(fb.focus_sinkhorn_bwd_workspace_bytes(shape, iters), dtype=torch.uint8, device="cuda")
+    dS = torch.empty_like(S)
+    fb.focus_sinkhorn_bwd(shape, S, tau, iters, ws, dG, dS)
+    d = dS[0].double()
+    size = d.abs().max().item()
+    assert d.sum(dim=0).abs().max().item() <= 1e-3 * size * n ** 0.5
+
+
 def test_sinkhorn_one_million_tokens():
     n, K, tau, iters = 1 << 20, 8, 0.1, 10
     g = torch.Generator(device="cuda"); g.manual_seed(8)
