@@ -34,8 +34,8 @@ UNIT = "TFLOP/s"
 
 # DRAM bytes per launch of the attention kernel (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture per
 # entry, see profiles/), keyed by (workload name, layout); only valid for the kernel sources with this digest.
-ATTN_TRAFFIC = {("M-llama3-8b-128k", 1): 6.425e9}
-ATTN_TRAFFIC_SOURCES = "edb12785400a8a17"
+ATTN_TRAFFIC = {("M-llama3-8b-128k", 1): 6.538e9}
+ATTN_TRAFFIC_SOURCES = "73736cfb1fef50ec"
 
 
 def attn_traffic(name, layout):
