@@ -295,6 +295,7 @@ def main():
     total_ms = t_start.elapsed_time(t_end)
     total_ms = multi.max_over_ranks(total_ms, dist, "cuda")
     assert status[0].item() == 0, f"kernel reported an expired wait: {status.tolist()}"
+    assert near.item() >= 0, "focus_assign set its fault flag (bit 63 of the near-tie word)"
     ms_step = total_ms / args.steps
     t_assign = float(np.mean([e[0].elapsed_time(e[1]) for e in marks]))
     t_tiles = float(np.mean([e[1].elapsed_time(e[2]) for e in marks]))

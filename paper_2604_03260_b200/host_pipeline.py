@@ -67,7 +67,8 @@ class HostPipeline:
     def run(self, hQ, hK, hV, hC, hO, hL):
         """One pass: pinned host tensors in (Q [Hq,n,D], K/V [Hkv,n,D] bf16, centroids [Hkv,K,D] fp32), pinned host
         tensors out (O bf16 [Hq,n,D], lse fp32 [Hq,n]).  Enqueues everything and makes the current stream wait for
-        both pipeline streams; it does not synchronise the host.  ``status[0]`` must read 0 afterwards."""
+        both pipeline streams; it does not synchronise the host.  Afterwards ``status[0]`` must read 0 and ``near``
+        (an int64 word: the near-tie count, bit 63 = fault flag of focus_assign) must not be negative."""
         G = self.G
         start = torch.cuda.Event()
         start.record()
