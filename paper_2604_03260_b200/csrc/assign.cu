@@ -4,7 +4,8 @@
 // The tiles of 128 vectors, numbered head by head, are dealt out as one contiguous range per block, a few blocks
 // per SM and all of them resident, so the launch is a single wave of equal shares.  The rows of a tile go to
 // shared memory with coalesced asynchronous 16-byte copies, laid out as the K-major, 128-byte-swizzled operand of
-// a tcgen05 MMA, two tiles in flight; whenever its range enters a head with another centroid set the block splits
+// a tcgen05 MMA, two tiles in flight (at D = 256 a tile travels as two pieces of 128 columns, so that three
+// blocks still fit an SM); whenever its range enters a head with another centroid set the block splits
 // those centroids into three bf16 terms each (hi + mid + lo carries 24 mantissa bits, so the products with the
 // bf16 vectors sum to the fp32 dot product) as the second operand.  Per tile one thread issues the MMA chain S = X C'^T (128 x 3K, fp32, in tensor
 // memory); while it runs every thread sums the squares of its own row from shared memory; then it reads its
@@ -23,7 +24,9 @@ template <int D, int KMAX>
 struct AssignCfg {
     static constexpr int NCOLS = (3 * KMAX + 15) / 16 * 16;             // rows of C' = columns of S
     static constexpr uint32_t SUB_BYTES = 128 * 128;                     // 128 vectors x 64 dimensions
-    static constexpr uint32_t TILE_BYTES = SUB_BYTES * (D / 64);
+    static constexpr int CW = D < 128 ? D : 128;                         // columns of a tile staged at a time (a "piece")
+    static constexpr int NP = D / CW;                                    // pieces per tile: 2 at D = 256
+    static constexpr uint32_t TILE_BYTES = SUB_BYTES * (CW / 64);        // one piece of one tile
     static constexpr uint32_t CSUB_BYTES = NCOLS * 128;                  // NCOLS rows x 64 dimensions
     static constexpr uint32_t C_BYTES = CSUB_BYTES * (D / 64);
     static constexpr uint32_t TMEM_COLS2 = 2 * NCOLS <= 32 ? 32 : (2 * NCOLS <= 64 ? 64 : (2 * NCOLS <= 128 ? 128 : 256));   // two S buffers
@@ -32,7 +35,7 @@ struct AssignCfg {
 };
 
 struct AssignCtl {
-    uint64_t s_full[2];               // the MMA chain of the tile in buffer 0 / 1 has completed
+    uint64_t s_full[2];               // the MMAs that read the piece in buffer 0 / 1 have completed
     uint32_t tmem_base;
     int fault;
     float cn2[32];                    // |c_g|^2, then 1/|c_g|
@@ -50,7 +53,8 @@ assign_kernel(const __nv_bfloat16* __restrict__ x, int64_t stride_b, int64_t str
     const uint32_t sc = base + 2 * Cfg::TILE_BYTES;            // centroid operand C'
     unsigned char* const cprime = sm + 2 * Cfg::TILE_BYTES;
     AssignCtl* const ctl = reinterpret_cast<AssignCtl*>(sm + 2 * Cfg::TILE_BYTES + Cfg::C_BYTES);
-    constexpr int CPR = D / 8;                                 // 16-byte chunks per row
+    constexpr int CW = Cfg::CW, NP = Cfg::NP;
+    constexpr int CPR = CW / 8;                                // 16-byte chunks per row of a piece
     constexpr int RSTEP = ASSIGN_THREADS / CPR;                // rows covered by one copy per thread
 
     // block i takes `share` items, the first `extra` blocks one more: items item0 .. item0 + T - 1 of the list
@@ -69,12 +73,13 @@ assign_kernel(const __nv_bfloat16* __restrict__ x, int64_t stride_b, int64_t str
     const __nv_bfloat16* const xrow0 = x + (size_t)r0 * stride_n + cc * 8;
     const size_t step = (size_t)RSTEP * stride_n;
     const uint32_t dst0 = sx + (cc >> 3) * Cfg::SUB_BYTES + r0 * 128;
-    auto copy_tile = [&](int t) {
-        if (t < T) {
+    auto copy_tile = [&](int q) {                               // q = piece number: tile q / NP, columns (q % NP) * CW ...
+        if (q < T * NP) {
+            const int t = q / NP, c = q % NP;
             const int bh = (item0 + t) / ntile, tok0 = ((item0 + t) % ntile) * 128;
-            const __nv_bfloat16* src = xrow0 + (size_t)(bh / H) * stride_b + (size_t)(bh % H) * stride_h + (size_t)tok0 * stride_n;
+            const __nv_bfloat16* src = xrow0 + (size_t)(bh / H) * stride_b + (size_t)(bh % H) * stride_h + (size_t)tok0 * stride_n + c * CW;
             const int left = n - tok0 - r0;                    // copy i is in range iff i * RSTEP < left
-            const uint32_t dstb = dst0 + (t & 1) * Cfg::TILE_BYTES;
+            const uint32_t dstb = dst0 + (q & 1) * Cfg::TILE_BYTES;
 #pragma unroll
             for (int i = 0; i < ASSIGN_THREADS / RSTEP; ++i) {
                 const uint32_t dst = dstb + i * RSTEP * 128 + ((((uint32_t)cc & 7u) ^ ((uint32_t)(r0 + (i * RSTEP) % 8) & 7u)) << 4);
@@ -139,8 +144,10 @@ assign_kernel(const __nv_bfloat16* __restrict__ x, int64_t stride_b, int64_t str
     uint32_t tmem = 0;
     unsigned int near_votes = 0;
     int cur_hk = -1;
-    for (int t = 0; t < T; ++t) {
-        const int buf = t & 1;
+    float2 a0 = make_float2(0.f, 0.f), a1 = make_float2(0.f, 0.f);      // |x|^2 of the thread's row, over the pieces
+    for (int q = 0; q < T * NP; ++q) {
+        const int t = q / NP, c = q % NP;                      // tile and piece
+        const int buf = q & 1, abuf = t & 1;                   // piece buffer, accumulator buffer
         const int bh = (item0 + t) / ntile, tile = (item0 + t) % ntile;
         const int hk = (bh % H) / G;
         if (hk != cur_hk) {
@@ -159,19 +166,19 @@ assign_kernel(const __nv_bfloat16* __restrict__ x, int64_t stride_b, int64_t str
                 const uint64_t xd = smem_desc_sw128(sx + buf * Cfg::TILE_BYTES, 16, 1024);
                 const uint64_t cd = smem_desc_sw128(sc, 16, 1024);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    umma_ss(tmem + buf * Cfg::NCOLS, xd + (uint64_t)(((ks / 4) * Cfg::SUB_BYTES + (ks % 4) * 32) >> 4),
-                            cd + (uint64_t)(((ks / 4) * Cfg::CSUB_BYTES + (ks % 4) * 32) >> 4), IDESC, ks > 0);
+                for (int ks = 0; ks < CW / 16; ++ks)
+                    umma_ss(tmem + abuf * Cfg::NCOLS, xd + (uint64_t)(((ks / 4) * Cfg::SUB_BYTES + (ks % 4) * 32) >> 4),
+                            cd + (uint64_t)(((c * (CW / 64) + ks / 4) * Cfg::CSUB_BYTES + (ks % 4) * 32) >> 4), IDESC,
+                            (c > 0 || ks > 0) ? 1u : 0u);
                 umma_commit(smem_u32(&ctl->s_full[buf]));
             }
             __syncwarp();
         }
         // ---- |x|^2 of the thread's own row while the MMAs run (packed fp32 pairs)
-        float xx;
         {
             const unsigned char* row = sm + buf * Cfg::TILE_BYTES + threadIdx.x * 128;
             const uint32_t sw = (threadIdx.x & 7u) << 4;
-            float2 a0 = make_float2(0.f, 0.f), a1 = make_float2(0.f, 0.f);
+            if (c == 0) a0 = a1 = make_float2(0.f, 0.f);
 #pragma unroll
             for (int v = 0; v < CPR; ++v) {
                 const uint4 rv = *reinterpret_cast<const uint4*>(row + (v >> 3) * Cfg::SUB_BYTES + ((((uint32_t)v & 7u) << 4) ^ sw));
@@ -182,30 +189,32 @@ assign_kernel(const __nv_bfloat16* __restrict__ x, int64_t stride_b, int64_t str
                 a0 = __ffma2_rn(v0, v0, a0); a1 = __ffma2_rn(v1, v1, a1);
                 a0 = __ffma2_rn(v2, v2, a0); a1 = __ffma2_rn(v3, v3, a1);
             }
-            xx = (a0.x + a0.y) + (a1.x + a1.y);
         }
-        if (ok && !mbar_wait(smem_u32(&ctl->s_full[buf]), (uint32_t)((t >> 1) & 1))) {
+        const float xx = (a0.x + a0.y) + (a1.x + a1.y);
+        const bool last_piece = c == NP - 1;
+        if (ok && !mbar_wait(smem_u32(&ctl->s_full[buf]), (uint32_t)((q >> 1) & 1))) {
             ok = false;
             ctl->fault = 1;
         }
         tc_fence_after();
         float sc3[Cfg::NCOLS];
-        if (ok) {
+        if (ok && last_piece) {
 #pragma unroll
-            for (int c = 0; c < Cfg::NCOLS / 16; ++c) {
+            for (int cc16 = 0; cc16 < Cfg::NCOLS / 16; ++cc16) {
                 uint32_t v[16];
-                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + buf * Cfg::NCOLS + c * 16, v);
+                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + abuf * Cfg::NCOLS + cc16 * 16, v);
                 tmem_wait_ld();
 #pragma unroll
-                for (int e = 0; e < 16; ++e) sc3[c * 16 + e] = __uint_as_float(v[e]);
+                for (int e = 0; e < 16; ++e) sc3[cc16 * 16 + e] = __uint_as_float(v[e]);
             }
         } else {
 #pragma unroll
             for (int e = 0; e < Cfg::NCOLS; ++e) sc3[e] = 0.f;
         }
         tc_fence_before();
-        __syncthreads();                                       // the tile's buffer is free: its MMAs and every row sum are done
-        copy_tile(t + 2);
+        __syncthreads();                                       // the piece's buffer is free: its MMAs and every row sum are done
+        copy_tile(q + 2);
+        if (!last_piece) continue;
 
         const int tok = tile * 128 + threadIdx.x;
         const bool in = tok < n;
