@@ -18,7 +18,7 @@ constexpr float DEC_LOG2E = 1.4426950408889634f;
 constexpr float DEC_LN2 = 0.6931471805599453f;
 
 template <int D> struct DecCfg {
-    static constexpr int WARPS = 4;                                // warps per CTA: two CTAs per SM at D <= 128, one at D = 256
+    static constexpr int WARPS = D == 256 ? 2 : 4;                 // warps per CTA: two CTAs fit an SM at every D
     static constexpr int ROWB = 2 * D + 16;                        // padded row: conflict-free ldmatrix rows
     static constexpr int STAGE = 2 * DEC_GK * ROWB;                // K rows then V rows of one step
     static constexpr size_t SMEM = (size_t)WARPS * DEC_NST * STAGE;
@@ -283,7 +283,7 @@ decode_merge_kernel(const float* __restrict__ part, int nsplit, int D, int Hq, _
     if (t == 0) lse[hq] = (M + log2f(L)) * DEC_LN2;
 }
 
-static int decode_warps(int) { return 4; }
+static int decode_warps(int D) { return D == 256 ? 2 : 4; }
 
 static int decode_splits(const focus_shape* s) {
     const int groups = cdiv(s->n, DEC_GK);
