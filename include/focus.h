@@ -396,13 +396,31 @@ FOCUS_API int focus_selftest_stalled_wait(const focus_shape* shape, focus_tensor
 
 /*
  * focus_selftest_umma_pair -- diagnostic (the paper has no counterpart): the same two tiles with D = 128 through one
- * MMA shared by a pair of CTAs on neighbouring SMs, the form focus_attn_fwd uses at D = 128: 256 rows of A and P (128
+ * MMA shared by a pair of CTAs on neighbouring SMs (a form focus_attn_fwd does not use): 256 rows of A and P (128
  * per CTA), each CTA staging half of B (64 of its 128 rows) and half of V (64 of its 128 columns).
  *   a, p      device bf16 [256, 128] row-major     b, v   device bf16 [128, 128] row-major
  *   s_out, o_out   device fp32 [256, 128]          dev_status   as above
  */
 FOCUS_API int focus_selftest_umma_pair(const void* a, const void* b, const void* p, const void* v, float* s_out,
                                        float* o_out, int32_t* dev_status, void* stream);
+
+/*
+ * focus_selftest_mma_rate -- diagnostic (the paper has no counterpart): the rate at which the tensor pipe works off
+ * tcgen05 MMAs when nothing else runs, in the shapes the attention kernel uses or could use.  One CTA (pair = 0) or CTA
+ * pair (pair = 1, M = 256) per SM issues `rounds` rounds of MMA chains on operands resident in shared and tensor
+ * memory; a chain is eight K = 16 instructions = one 128 x N x 128 product (256 x N x 128 across a pair).
+ *   N         64, 96, 128 or 256 (pairs: 128 or 256)
+ *   ts        0: both operands from shared memory, K-major (S = Q K^T); 1: A from tensor memory, B MN-major (O = P V), N <= 128
+ *   pattern   0: one chain per commit, two commits in flight; 1: two chains of the first form per commit, instructions
+ *             alternating; 2: one chain of each form per commit, alternating; 3: one of each, one after the other
+ *             (patterns 1-3: four chains in flight, ts = 0, N <= 128)
+ *   rounds    2 ... 1000000
+ *   result    device, three 64-bit words, written by CTA 0: clock cycles, nanoseconds, fault flag (1 if a wait of the
+ *             probe ran out after 1 s; the kernel then drains and returns)
+ * flop per clock and SM = chains per round x 2 x 128 x N x 128 x rounds / cycles (nominal bf16 rate: 8192).
+ */
+FOCUS_API int focus_selftest_mma_rate(int32_t pair, int32_t N, int32_t ts, int32_t pattern, int32_t rounds,
+                                      unsigned long long* result, void* stream);
 
 #ifdef __cplusplus
 }

@@ -106,6 +106,8 @@ def lib():
         L.focus_selftest_umma.argtypes = [i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.focus_selftest_umma_pair.restype = C.c_int
         L.focus_selftest_umma_pair.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+        L.focus_selftest_mma_rate.restype = C.c_int
+        L.focus_selftest_mma_rate.argtypes = [i32, i32, i32, i32, i32, vp, vp]
         L.focus_selftest_stalled_wait.restype = C.c_int
         L.focus_selftest_stalled_wait.argtypes = [SP, focus_tensor, focus_tensor, focus_tensor, focus_tensor, vp, C.c_uint64, vp, vp]
         _lib = L
@@ -252,6 +254,11 @@ def focus_selftest_umma(D, a, b, p, v, s_out, o_out, dev_status, stream=None):
 
 def focus_selftest_umma_pair(a, b, p, v, s_out, o_out, dev_status, stream=None):
     _check(lib().focus_selftest_umma_pair(_p(a), _p(b), _p(p), _p(v), _p(s_out), _p(o_out), _p(dev_status), _stream(stream)))
+
+
+def focus_selftest_mma_rate(pair, N, ts, pattern, rounds, result, stream=None):
+    """result: int64 device tensor of 3 words (cycles, nanoseconds, fault flag)"""
+    _check(lib().focus_selftest_mma_rate(pair, N, ts, pattern, rounds, _p(result), _stream(stream)))
 
 
 def focus_selftest_stalled_wait(shape, q, k, v, o, lse, wait_limit_ns, dev_status, stream=None):

@@ -262,6 +262,158 @@ static int run_pair_selftest(const void* a, const void* b, const void* p, const 
     return check_cuda(cudaGetLastError(), "pair selftest launch");
 }
 
+
+// ---- focus_selftest_mma_rate: what the tensor pipe delivers when it is fed nothing but MMAs, in the shapes the attention
+// kernel uses or could use.  One CTA (or CTA pair) per SM, operands resident in shared and tensor memory (pseudo-random
+// finite bf16 values, so that the datapath switches as on real data), chains of eight K = 16 instructions (one
+// 128 x N x 128 product, or 256 x N x 128 across a pair).  `pattern` 0: one chain per commit, two commits in flight;
+// 1: two S-type chains per commit, issued alternately; 2: an S-type and a P V-type chain per commit, issued alternately;
+// 3: an S-type chain, then a P V-type chain, per commit (four chains in flight in patterns 1-3).
+template <int PAIR, int TS, int PATTERN>
+__global__ void __launch_bounds__(128) mma_rate_kernel(int N, int rounds, unsigned long long* res) {
+    constexpr int ts = TS, pattern = PATTERN;
+    using namespace ptx;
+    extern __shared__ __align__(1024) unsigned char sm[];
+    __shared__ __align__(8) uint64_t bars[2];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int fault_s;
+    const uint32_t base = smem_u32(sm);
+    const int warp = threadIdx.x >> 5;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0;
+    const uint32_t sa = base, sb = base + 32768;              // A: 128 rows x 128 K; B: up to 256 rows x 128 K (or V: 128 keys x N)
+    for (uint32_t i = threadIdx.x; i < (32768u + 65536u) / 4; i += 128) {
+        uint32_t x = (i + 1u) * 2654435761u + blockIdx.x * 40503u;
+        x ^= x >> 15; x *= 2246822519u; x ^= x >> 13;
+        const uint32_t lo = 0x3c00u | (x & 0x83ffu), hi = 0x3c00u | ((x >> 16) & 0x83ffu);   // finite, |v| in [2^-7, 2)
+        reinterpret_cast<uint32_t*>(sm)[i] = lo | (hi << 16);
+    }
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars[0]), 1);
+        mbar_init(smem_u32(&bars[1]), 1);
+        fence_mbar_init();
+        fault_s = 0;
+    }
+    if (warp == 0) {
+        if (PAIR) { tmem_alloc_pair(smem_u32(&tmem_base_s), 512); tmem_relinquish_pair(); }
+        else { tmem_alloc(smem_u32(&tmem_base_s), 512); tmem_relinquish(); }
+    }
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    if (PAIR) cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+    constexpr uint32_t COL_P = 448;                             // the A operand of the TS form: 64 columns of packed bf16 pairs
+    if (ts || pattern >= 2) {
+        uint32_t r[32];
+        for (int c = 0; c < 32; ++c) r[c] = 0x3c003c00u + (uint32_t)(c * 65537u + threadIdx.x);
+        tmem_st32(tmem + ((uint32_t)(warp * 32) << 16) + COL_P, r);
+        tmem_st32(tmem + ((uint32_t)(warp * 32) << 16) + COL_P + 32, r);
+        tmem_wait_st();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (PAIR) cluster_sync_all();
+    tc_fence_after();
+    if (rank == 0 && warp == 0) {
+        if (elect_one()) {
+            const uint32_t M = PAIR ? 256 : 128;
+            const uint32_t idesc_ss = idesc_bf16(M, N, 0, 0), idesc_ts = idesc_bf16(M, N, 0, 1);
+            const uint32_t bsub = (PAIR ? N / 2 : N) * 128;      // bytes of a 64-column sub-tile of the K-major B operand
+            const uint32_t vlbo = 128 * 128;                      // MN-major B: 64-column groups 16 KB apart
+            // descriptors once, so that the loop below is nothing but the MMAs
+            uint64_t adesc[8], bdesc[8], vdesc[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                adesc[k] = smem_desc_sw128(sa + (k / 4) * 16384 + (k % 4) * 32, 16, 1024);
+                bdesc[k] = smem_desc_sw128(sb + (k / 4) * bsub + (k % 4) * 32, 16, 1024);
+                vdesc[k] = smem_desc_sw128(sb + k * 2048, vlbo, 1024);
+            }
+            auto ss = [&](uint32_t d, int k, bool acc) {
+                if (PAIR) umma_ss_pair(d, adesc[k], bdesc[k], idesc_ss, acc); else umma_ss(d, adesc[k], bdesc[k], idesc_ss, acc);
+            };
+            auto tsf = [&](uint32_t d, int k, bool acc) {
+                if (PAIR) umma_ts_pair(d, tmem + COL_P + k * 8, vdesc[k], idesc_ts, acc); else umma_ts(d, tmem + COL_P + k * 8, vdesc[k], idesc_ts, acc);
+            };
+            auto wait_round = [&](int r) -> bool {                // the commit of round r has arrived (bounded)
+                const uint64_t w0 = globaltimer_ns();
+                while (!mbar_try_wait(smem_u32(&bars[r & 1]), (uint32_t)((r >> 1) & 1)))
+                    if (globaltimer_ns() - w0 > 1000000000ull) return false;
+                return true;
+            };
+            const unsigned long long c0 = clock64(), t0 = globaltimer_ns();
+            bool ok = true;
+            for (int r = 0; r < rounds && ok; ++r) {
+                const int b = r & 1;
+                if (r >= 2 && !wait_round(r - 2)) { ok = false; break; }
+                if (pattern == 0) {
+                    const uint32_t d = tmem + (uint32_t)b * (uint32_t)N;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) { if (ts) tsf(d, k, k > 0); else ss(d, k, k > 0); }
+                } else {
+                    // two chains per round; with P in the way (patterns 2, 3 at N = 128) both rounds share one pair of accumulators
+                    const uint32_t d0 = tmem + ((pattern >= 2 && 4 * N > (int)COL_P) ? 0u : (uint32_t)b * 2u * (uint32_t)N), d1 = d0 + (uint32_t)N;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const int which = pattern == 3 ? i / 8 : i & 1, k = pattern == 3 ? i % 8 : i / 2;
+                        if (which == 1 && pattern >= 2) tsf(d1, k, k > 0);
+                        else ss(which ? d1 : d0, k, k > 0);
+                    }
+                }
+                if (PAIR) umma_commit_pair(smem_u32(&bars[b])); else umma_commit(smem_u32(&bars[b]));
+            }
+            for (int r = rounds - 2; r < rounds && ok; ++r)
+                if (r >= 0 && !wait_round(r)) ok = false;
+            const unsigned long long c1 = clock64(), t1 = globaltimer_ns();
+            if (!ok) fault_s = 1;
+            if (blockIdx.x == 0) { res[0] = c1 - c0; res[1] = t1 - t0; }
+            if (!ok) res[2] = 1;
+        }
+        __syncwarp();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (PAIR) cluster_sync_all();
+    if (fault_s) { const uint64_t w0 = globaltimer_ns(); while (globaltimer_ns() - w0 < 20000ull) { } }
+    if (warp == 0) { if (PAIR) tmem_dealloc_pair(tmem, 512); else tmem_dealloc(tmem, 512); }
+}
+
+static int run_mma_rate(int pair, int N, int ts, int pattern, int rounds, unsigned long long* res, cudaStream_t st) {
+    int rc, dev = 0, sms = 0;
+    if ((rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice"))) return rc;
+    if ((rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "cudaDeviceGetAttribute"))) return rc;
+    const size_t smem = 32768 + 65536;
+    if ((rc = check_cuda(cudaMemsetAsync(res, 0, 3 * sizeof(unsigned long long), st), "cudaMemsetAsync(mma rate)"))) return rc;
+    auto launch = [&](auto kern) -> int {
+        int r2 = check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem), "cudaFuncSetAttribute(mma rate)");
+        if (r2) return r2;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(pair ? (unsigned)(sms / 2) * 2 : (unsigned)sms); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = pair ? 2 : 1; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        return check_cuda(cudaLaunchKernelEx(&cfg, kern, N, rounds, res), "mma rate launch");
+    };
+    if (pair) {
+        switch (pattern) {
+            case 0: rc = ts ? launch(mma_rate_kernel<1, 1, 0>) : launch(mma_rate_kernel<1, 0, 0>); break;
+            case 1: rc = launch(mma_rate_kernel<1, 0, 1>); break;
+            case 2: rc = launch(mma_rate_kernel<1, 0, 2>); break;
+            default: rc = launch(mma_rate_kernel<1, 0, 3>); break;
+        }
+    } else {
+        switch (pattern) {
+            case 0: rc = ts ? launch(mma_rate_kernel<0, 1, 0>) : launch(mma_rate_kernel<0, 0, 0>); break;
+            case 1: rc = launch(mma_rate_kernel<0, 0, 1>); break;
+            case 2: rc = launch(mma_rate_kernel<0, 0, 2>); break;
+            default: rc = launch(mma_rate_kernel<0, 0, 3>); break;
+        }
+    }
+    if (rc) return rc;
+    return check_cuda(cudaGetLastError(), "mma rate launch");
+}
+
 }  // namespace focus
 
 extern "C" int focus_selftest_umma(int32_t D, const void* a, const void* b, const void* p, const void* v, float* s_out,
@@ -285,4 +437,21 @@ extern "C" int focus_selftest_umma_pair(const void* a, const void* b, const void
     int rc = require_sm100();
     if (rc) return rc;
     return run_pair_selftest(a, b, p, v, s_out, o_out, dev_status, (cudaStream_t)stream);
+}
+
+extern "C" int focus_selftest_mma_rate(int32_t pair, int32_t N, int32_t ts, int32_t pattern, int32_t rounds,
+                                       unsigned long long* result, void* stream) {
+    using namespace focus;
+    if (!result) return fail(FOCUS_ERR_INVALID_ARG, "result is NULL");
+    if (pair < 0 || pair > 1 || ts < 0 || ts > 1 || pattern < 0 || pattern > 3 || rounds < 2 || rounds > 1000000)
+        return fail(FOCUS_ERR_INVALID_ARG, "pair, ts in {0, 1}, pattern in 0..3, rounds in 2..1000000");
+    if (N != 64 && N != 96 && N != 128 && N != 256) return fail(FOCUS_ERR_INVALID_ARG, "N must be 64, 96, 128 or 256");
+    // tensor memory: two (pattern 0) or four accumulators of N columns, plus 64 columns of P for the TS form
+    if ((ts || pattern >= 2) && N > 128) return fail(FOCUS_ERR_INVALID_ARG, "the TS form takes N <= 128 here");
+    if (pattern == 1 && N > 128) return fail(FOCUS_ERR_INVALID_ARG, "two interleaved chains per commit take N <= 128 here");
+    if (pattern >= 1 && ts) return fail(FOCUS_ERR_INVALID_ARG, "patterns 1-3 fix the forms of their chains: pass ts = 0");
+    if (pair && N < 128) return fail(FOCUS_ERR_INVALID_ARG, "the CTA-pair form takes N = 128 or 256 here");
+    int rc = require_sm100();
+    if (rc) return rc;
+    return run_mma_rate(pair, N, ts, pattern, rounds, result, (cudaStream_t)stream);
 }

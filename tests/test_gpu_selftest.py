@@ -67,3 +67,25 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(D):
     masks = np.full((wl.Hq, wl.n), 0b11, np.uint32), np.full((wl.Hkv, wl.n), 0b11, np.uint32)
     O2, lse2 = gpu_attn(wl, Q, K, V)                # asserts a clean status itself
     assert_parity(compare_rows(wl, Q, K, V, masks[0], masks[1], O2, lse2, dense=True))
+
+
+@pytest.mark.parametrize("pair,N,ts,pattern", [(0, 128, 0, 0), (0, 128, 1, 0), (0, 256, 0, 0), (1, 128, 0, 0), (1, 128, 1, 0),
+                                               (0, 128, 0, 1), (0, 128, 0, 3), (1, 128, 0, 3), (0, 64, 0, 2), (0, 96, 0, 3)])
+def test_mma_rate_probe_runs_and_reports_a_plausible_rate(pair, N, ts, pattern):
+    """the probe's waits end, and the rate it reports lies between a tenth of and a little above the nominal one"""
+    rounds = 500
+    res = torch.full((3,), -1, dtype=torch.int64, device="cuda")
+    fb.focus_selftest_mma_rate(pair, N, ts, pattern, rounds, res)
+    torch.cuda.synchronize()
+    cycles, ns, fault = (int(x) for x in res.tolist())
+    assert fault == 0 and cycles > 0 and ns > 0
+    chains = 1 if pattern == 0 else 2
+    rate = chains * 2.0 * 128 * N * 128 * rounds / cycles
+    assert 0.1 * 8192 < rate < 1.05 * 8192, rate
+
+
+def test_mma_rate_probe_refuses_shapes_without_room_in_tensor_memory():
+    res = torch.zeros(3, dtype=torch.int64, device="cuda")
+    for args in ((0, 256, 1, 0), (0, 256, 0, 1), (1, 64, 0, 0), (0, 128, 1, 2), (0, 100, 0, 0)):
+        with pytest.raises(fb.FocusError):
+            fb.focus_selftest_mma_rate(*args, 100, res)
