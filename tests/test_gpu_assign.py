@@ -44,6 +44,16 @@ def test_assign_shapes(D, K, t, n):
     check(wl, Kt, C.contiguous(), wl.Hkv)
 
 
+@pytest.mark.parametrize("Hq,Hkv,D,n,K,t", [(64, 16, 128, 2048 + 77, 4, 2), (32, 8, 256, 3000, 8, 2), (96, 48, 64, 1500, 16, 3)])
+def test_assign_ranges_that_cross_heads(Hq, Hkv, D, n, K, t):
+    """more tiles than resident blocks and few tiles per head: a block's range of tiles runs through several heads and
+    KV heads, so it rebuilds its centroid operand on the way (at D = 256 with two pieces per tile)"""
+    wl = fi.Workload("x", Hq, Hkv, D, n, K, t, 8, seed=Hq + D + n)
+    Q, Kt, V, C = fi.make_inputs(wl, "cuda")
+    check(wl, Q, C, wl.Hq)
+    check(wl, Kt, C, wl.Hkv)
+
+
 @pytest.mark.parametrize("name", ["cfg3", "cfg4", "M128k", "cfg5"])
 def test_assign_large_configs_at_full_size(name):
     """every mask of the large configurations (clustered K = 8 at 32K, D = 256 top-1 at 64K, the 128K metric point,
