@@ -24,7 +24,9 @@ def hidden_inputs(n, d, dg, K, seed, batch=1):
 
 @pytest.mark.parametrize("n,d,dg,K,t,use_bias,batch", [(1, 64, 16, 4, 2, False, 1), (300, 768, 16, 4, 2, True, 1),
                                                        (5000, 4096, 16, 8, 2, True, 1), (1000, 200, 7, 5, 1, False, 2),
-                                                       (777, 1032, 32, 32, 3, True, 1), (129, 8, 4, 2, 2, False, 3)])
+                                                       (777, 1032, 32, 32, 3, True, 1), (129, 8, 4, 2, 2, False, 3),
+                                                       # more tiles than resident blocks: a block's range runs from one sequence into the next
+                                                       (8000, 520, 16, 4, 2, True, 8)])
 def test_masks_match_the_oracle(n, d, dg, K, t, use_bias, batch):
     Hq, Hkv = 4, 2
     h, Wg, C, bias = hidden_inputs(n, d, dg, K, n + d, batch)
